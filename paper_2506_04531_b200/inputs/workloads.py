@@ -1,0 +1,76 @@
+"""The synthetic workloads: a parameter layout, a cluster shape and an arrival trace each.
+
+They stand in for the paper's simulated geo-distributed cluster (four regions, heterogeneous
+worker speeds, profiled step times of Pythia-70M/160M/410M on one H100: 238.4, 623.0 and
+1589.7 ms) -- only the structure that reaches the server-side update path is kept.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List
+
+import numpy as np
+
+from . import gen
+from .layouts import Layout, named_layout
+from .trace import TraceSpec, generate_trace, worker_speeds
+
+
+@dataclass
+class Workload:
+    name: str
+    layout: Layout
+    n_workers: int
+    n_lps: int
+    worker_dtype: int
+    t_profiled_ms: float
+    n_arrivals: int
+    seed: int
+    K: int = 32
+    eta_l: float = 0.2
+    beta_l: float = 0.9
+    eta_g: float = 0.15
+    beta_g: float = 0.5
+    alpha: float = 0.25
+    slow_region_factor: float = 1.0   # speeds of the last region's workers are divided by this
+
+    @property
+    def worker_lps(self) -> List[int]:
+        per = self.n_workers // self.n_lps
+        return [w // per for w in range(self.n_workers)]
+
+    @property
+    def speeds(self) -> List[float]:
+        s = worker_speeds(self.n_workers, self.seed)
+        if self.slow_region_factor != 1.0:
+            wl = self.worker_lps
+            s = [v / self.slow_region_factor if wl[w] == self.n_lps - 1 else v for w, v in enumerate(s)]
+        return s
+
+    def trace(self, n_arrivals: int | None = None) -> np.ndarray:
+        return generate_trace(TraceSpec(
+            P=self.layout.P, worker_lps=self.worker_lps, speeds=self.speeds,
+            t_profiled_ms=self.t_profiled_ms, n_arrivals=n_arrivals or self.n_arrivals, K=self.K))
+
+    def hyper(self) -> dict:
+        return dict(eta_l=self.eta_l, beta_l=self.beta_l, eta_g=self.eta_g, beta_g=self.beta_g,
+                    alpha=self.alpha, K=self.K)
+
+
+def workload(name: str) -> Workload:
+    """toy | toy_k4 | 70m | 160m | 410m  (hyperparameters: the paper's selected values)."""
+    if name == "toy":
+        return Workload("toy", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1)
+    if name == "toy_k4":
+        return Workload("toy_k4", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1, K=4)
+    if name == "70m":
+        return Workload("70m", named_layout("70m"), 8, 2, gen.BF16, 238.4, 1000, seed=2)
+    if name == "160m":
+        return Workload("160m", named_layout("160m"), 16, 4, gen.F32, 623.0, 2000, seed=3)
+    if name == "410m":
+        return Workload("410m", named_layout("410m"), 32, 4, gen.F32, 1589.7, 2000, seed=4,
+                        slow_region_factor=3.0)
+    raise KeyError(name)
+
+
+SWEEP_SIZES = (1 << 20, 1 << 22, 1 << 24, 1 << 26, 70_426_624, 162_322_944, 1 << 28, 405_334_016, 1 << 30)

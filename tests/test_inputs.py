@@ -1,0 +1,125 @@
+"""Host-side checks of the synthetic input generators: layouts, noise, traces."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_2506_04531_b200.inputs import gen, layouts, trace as tr, workloads
+
+
+def test_layout_sizes():
+    want = {"70m": (70_426_624, 76), "160m": (162_322_944, 148), "410m": (405_334_016, 292),
+            "1p4b": (1_414_647_808, 292), "toy": (1 << 20, 1)}
+    for name, (P, n) in want.items():
+        lay = layouts.named_layout(name)
+        assert (lay.P, lay.n_tensors) == (P, n)
+        assert lay.offsets[-1] == P and len(lay.offsets) == n + 1
+    lay = layouts.named_layout("160m")
+    d, L, V = 768, 12, 50304
+    assert lay.P == 2 * V * d + L * (12 * d * d + 13 * d) + 2 * d
+    assert lay.tensors[0].name == "embed_in" and lay.tensors[-1].name == "embed_out"
+    assert min(t.numel for t in lay.tensors) == 768
+
+
+def test_noise_statistics_and_slicing():
+    key = gen.stream_key(5, gen.STREAM_WORKER + 3, 17)
+    z = gen.unit_noise(key, 0, 1 << 20)
+    assert z.dtype == np.float32
+    assert abs(float(z.mean())) < 5e-3
+    assert abs(float(z.var()) - 1.0) < 5e-3
+    assert float(np.abs(z).max()) <= 4.9
+    # kurtosis of Irwin-Hall(8) is 3 - 1.2/8 = 2.85
+    assert abs(float(((z.astype(np.float64)) ** 4).mean()) - 2.85) < 0.05
+    np.testing.assert_array_equal(gen.unit_noise(key, 12345, 23456), z[12345:23456])
+    # different streams / rounds / seeds decorrelate
+    z2 = gen.unit_noise(gen.stream_key(5, gen.STREAM_WORKER + 3, 18), 0, 1 << 16)
+    z3 = gen.unit_noise(gen.stream_key(5, gen.STREAM_WORKER + 4, 17), 0, 1 << 16)
+    for other in (z2, z3):
+        assert abs(float(np.corrcoef(z[: 1 << 16], other)[0, 1])) < 0.02
+    # neighbouring indices decorrelate
+    assert abs(float(np.corrcoef(z[:-1], z[1:])[0, 1])) < 5e-3
+
+
+def test_theta_init_per_tensor_rules():
+    lay = layouts.decoder_layout("tiny", 2, 16, 64)
+    th = gen.theta_init(lay, 3)
+    off = lay.offsets.astype(int)
+    for k, t in enumerate(lay.tensors):
+        seg = th[off[k]:off[k + 1]]
+        if t.kind == layouts.KIND_NORM_WEIGHT:
+            assert np.all(seg == 1.0)
+        elif t.kind == layouts.KIND_BIAS:
+            assert np.all(seg == 0.0)
+        else:
+            assert 0.015 < float(seg.std()) < 0.025
+    np.testing.assert_array_equal(gen.theta_init(lay, 3, 100, 3000), th[100:3000])
+
+
+def test_worker_result_dtypes_and_scales():
+    lay = layouts.decoder_layout("tiny", 1, 32, 128)
+    th = gen.theta_init(lay, 1)
+    r = gen.worker_result(th, lay, 1, 2, 0)
+    d = r.astype(np.float64) - th
+    off = lay.offsets.astype(int)
+    assert 0.8e-3 < d[off[0]:off[1]].std() < 1.2e-3          # matrix
+    assert 0.5e-4 < d[off[1]:off[2]].std() < 1.5e-4          # 1-D tensor
+    hb = gen.f32_to_bf16_bits(th)
+    rb = gen.worker_result(hb, lay, 1, 2, 0, worker_dtype=gen.BF16)
+    assert rb.dtype == np.uint16
+    lo, hi = 777, 2222
+    np.testing.assert_array_equal(gen.worker_result(hb[lo:hi], lay, 1, 2, 0, lo, hi, gen.BF16), rb[lo:hi])
+    # numpy bf16 helpers against the library conversion
+    import torch
+    x = (np.random.default_rng(0).normal(size=4096) * 0.02).astype(np.float32)
+    lib = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(gen.f32_to_bf16_bits(x), lib)
+    np.testing.assert_array_equal(gen.bf16_bits_to_f32(lib), torch.from_numpy(x).to(torch.bfloat16).float().numpy())
+
+
+@pytest.mark.parametrize("name", ["toy", "toy_k4", "70m", "160m", "410m"])
+def test_trace_structure(name):
+    wl = workloads.workload(name)
+    ev = wl.trace()
+    kinds = ev["kind"]
+    assert int((kinds == tr.ARRIVE).sum()) == wl.n_arrivals
+    t = ev["time_ns"]
+    assert np.all(np.diff(t) >= 0)
+    # replay the counters: pushes fire exactly on windows of K, each LPS alternates G and P
+    n_lps = wl.n_lps
+    tt, tl, phase = [0] * n_lps, [0] * n_lps, [0] * n_lps
+    n_push = 0
+    for e in ev:
+        k, l = int(e["kind"]), int(e["lps"])
+        if k == tr.ARRIVE:
+            assert wl.worker_lps[int(e["worker"])] == l
+            tt[l] += 1
+            if tt[l] - tl[l] == wl.K:
+                assert phase[l] == 0
+                phase[l] = 1
+                n_push += 1
+        elif k == tr.GPS_RECV:
+            assert phase[l] == 1
+            phase[l] = 2
+        else:
+            assert phase[l] == 2
+            phase[l] = 0
+            tl[l] = tt[l]
+    assert all(p == 0 for p in phase)                     # in-flight round trips were drained
+    assert int((kinds == tr.GPS_RECV).sum()) == n_push == int((kinds == tr.PULL).sum())
+    if name != "toy":
+        assert n_push >= 8
+    # regenerating gives the same trace
+    np.testing.assert_array_equal(ev, wl.trace())
+
+
+def test_trace_heterogeneity():
+    wl = workloads.workload("410m")
+    ev = wl.trace()
+    s = wl.speeds
+    assert 1.0 / 3.0 <= min(s) and max(s) <= 4.0
+    arr = ev[ev["kind"] == tr.ARRIVE]
+    per_lps = [int((arr["lps"] == l).sum()) for l in range(4)]
+    assert per_lps[3] < min(per_lps[:3])                  # the slowed-down region arrives least often
+    # a worker's arrivals are evenly spaced by its round time
+    w0 = arr[arr["worker"] == 0]["time_ns"]
+    assert len(set(np.diff(w0).tolist())) == 1
