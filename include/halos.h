@@ -1,0 +1,225 @@
+/* halos.h -- C ABI of the B200 (sm_100a) server-side update path of HALoS
+ * (hierarchical asynchronous local SGD).
+ *
+ * One context holds, on ONE GPU, the state of one global parameter server (GPS), n_lps local
+ * parameter servers (LPS) and n_workers workers over P fp32 master parameters:
+ *
+ *   GPS     Theta (global model), m_g (global momentum), i (GPS iteration)
+ *   LPS l   theta (local model), m_l (local momentum), anchor (theta_{t_last}),
+ *           outbox (Delta travelling to the GPS), inbox (Theta_i travelling back), t, t_last
+ *   worker  theta0 (theta_{t,0}: the model it was last scheduled with), in worker_dtype
+ *
+ * Every call maps to lines of Algorithm 1 ("HALoS Update Rules") of the paper; ModelUpdate is
+ * the momentum rule of Appendix E (update rules of the LPS and the GPS) applied to a
+ * displacement d:   m' = beta m + d ;   x' = x + eta [ (1 - beta) d + beta m' ].
+ *
+ * Conventions
+ *  - All state buffers are flat, packed in tensor order (tensor k starts at the sum of the
+ *    sizes before it), fp32 except worker snapshots (worker_dtype).  The context OWNS them.
+ *  - Pointers named *_dev are device pointers on the context's device, *_host are host pointers.
+ *  - All device work is enqueued on the stream given at creation; calls are asynchronous and
+ *    stream ordered.  Host-side counters (t, t_last, i, phases) change at enqueue time.
+ *  - Every call returns a status; on any status other than HALOS_OK the context's state is
+ *    unchanged and out-parameters are not written.  Nothing aborts or traps.
+ *  - A context is not thread safe.  There is no CPU fallback: without a CUDA device
+ *    halos_create fails with HALOS_ERR_CUDA.
+ */
+#ifndef HALOS_H
+#define HALOS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct halos_ctx halos_ctx;
+
+enum {
+    HALOS_OK = 0,
+    HALOS_ERR_INVALID_ARG = 1,
+    HALOS_ERR_BAD_STATE = 2,   /* call order violates Algorithm 1 (e.g. pull before the GPS answered) */
+    HALOS_ERR_OOM = 3,
+    HALOS_ERR_CUDA = 4,
+    HALOS_ERR_UNSUPPORTED = 5
+};
+
+enum { HALOS_F32 = 0, HALOS_BF16 = 1 };
+
+/* flags */
+enum {
+    HALOS_FLAG_STATS = 1u          /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
+};
+
+/* LPS phase of the push / merge round trip */
+enum { HALOS_IDLE = 0, HALOS_PUSHED = 1, HALOS_ANSWERED = 2 };
+
+/* buffers addressable through halos_peek / halos_read */
+enum {
+    HALOS_BUF_THETA_G = 0,  /* Theta          (index ignored) */
+    HALOS_BUF_M_G = 1,      /* m_g            (index ignored) */
+    HALOS_BUF_THETA_L = 2,  /* theta  of LPS index */
+    HALOS_BUF_M_L = 3,      /* m_l    of LPS index */
+    HALOS_BUF_ANCHOR = 4,   /* theta_{t_last} of LPS index */
+    HALOS_BUF_OUTBOX = 5,   /* Delta in flight from LPS index */
+    HALOS_BUF_INBOX = 6,    /* Theta_i in flight to LPS index */
+    HALOS_BUF_THETA0 = 7    /* start snapshot of worker index (worker_dtype) */
+};
+
+typedef struct halos_config {
+    uint32_t struct_size;          /* = sizeof(halos_config); checked */
+    uint32_t n_lps;
+    uint32_t n_workers;
+    const uint32_t* worker_lps;    /* host, [n_workers]: LPS of each worker; copied */
+    uint32_t n_tensors;
+    const uint64_t* tensor_numel;  /* host, [n_tensors]: elements per tensor; copied; sum = P */
+    float eta_l, beta_l;           /* local learning rate and momentum  (paper's selection: 0.2, 0.9) */
+    float eta_g, beta_g;           /* global learning rate and momentum (0.15, 0.5) */
+    float alpha;                   /* merging weight (0.25) */
+    uint32_t K;                    /* local updates accumulated per push (32) */
+    uint32_t worker_dtype;         /* HALOS_F32 | HALOS_BF16: type of theta0 snapshots and theta_H inputs */
+    uint32_t flags;
+    int32_t device;                /* CUDA device ordinal */
+    void* stream;                  /* cudaStream_t; NULL = the legacy default stream */
+    /* Optional device allocator (e.g. a shim over the PyTorch caching allocator).  NULL = cudaMalloc /
+     * cudaFree.  alloc returns a device pointer aligned to >= 256 bytes or NULL. */
+    void* (*alloc)(size_t bytes, void* user);
+    void (*free_)(void* ptr, void* user);
+    void* alloc_user;
+    uint32_t chunk_elems;          /* scheduler chunk size in elements; 0 = library default */
+    uint32_t reserved;
+} halos_config;
+
+/* Fills *cfg with the paper's selected hyperparameters and library defaults (everything else zero). */
+void halos_default_config(halos_config* cfg);
+
+/* Alg. 1 lines 6-7 (initialisation): Theta = theta[l] = anchor[l] = Theta_0, theta0[w] = cast(Theta_0),
+ * momenta 0, t = t_last = i = 0.  theta_init_dev: device, P fp32, flat, borrowed during the call only
+ * (the call synchronises the stream before returning).  *out receives the context. */
+int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx** out);
+
+/* Alg. 1 line 25 (worker side, delta = theta_{t,H} - theta_{t,0}).  Registers the result theta_{t,H}
+ * of `worker`; the subtraction itself is fused into the next halos_lps_apply for this worker so
+ * delta never touches memory.  Exactly one of thetaH_flat_dev (device, P elements of worker_dtype,
+ * packed like the state) and thetaH_ptrs_host (host array of n_tensors DEVICE pointers, one per
+ * tensor, each tensor contiguous) is non-NULL.  The device data is BORROWED until the matching
+ * halos_lps_apply has completed in stream order.  BAD_STATE if the worker already has a pending
+ * result. */
+int halos_worker_delta(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_dev,
+                       const void* const* thetaH_ptrs_host);
+
+/* Same, for a result that sits in HOST memory (P elements of worker_dtype, packed): it is copied
+ * into a context-owned staging buffer on the stream (pinned host memory makes the copy
+ * asynchronous), so the borrow ends when that copy has completed in stream order. */
+int halos_worker_delta_host(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_host);
+
+/* Alg. 1 lines 10-13 at LPS `lps` for the pending result of `worker`:  t <- t+1;
+ * theta_t <- ModelUpdate(theta_{t-1}, delta, eta_l, beta_l); the worker is scheduled theta_t
+ * (theta0[worker] <- cast(theta_t)).  One fused kernel.  *push_due (may be NULL) receives
+ * (t - t_last == K).  INVALID_ARG if the worker does not belong to lps; BAD_STATE if it has no
+ * pending result. */
+int halos_lps_apply(halos_ctx* ctx, uint32_t lps, uint32_t worker, int* push_due);
+
+/* Alg. 1 line 14: outbox[lps] <- Delta = theta_t - theta_{t_last}.  The LPS goes on updating while
+ * Delta is in flight.  BAD_STATE if a round trip is already in flight for this LPS.  The library
+ * does not insist on t - t_last == K; the caller (halos_replay) decides when to push. */
+int halos_lps_push(halos_ctx* ctx, uint32_t lps);
+
+/* Alg. 1 lines 2-4: the GPS receives outbox[lps]; i <- i+1; Theta_i <- ModelUpdate(Theta_{i-1}, Delta,
+ * eta_g, beta_g); inbox[lps] <- Theta_i (a snapshot).  BAD_STATE unless lps has pushed. */
+int halos_gps_merge(halos_ctx* ctx, uint32_t lps);
+
+/* Alg. 1 lines 18-19: t_last <- t; theta_t <- (1-alpha) theta_t + alpha inbox[lps]; anchor <- theta_t.
+ * BAD_STATE unless the GPS has answered this LPS. */
+int halos_lps_pull(halos_ctx* ctx, uint32_t lps);
+
+/* Synchronises the stream and frees everything the context owns.  NULL is accepted. */
+int halos_destroy(halos_ctx* ctx);
+
+/* ------------------------------------------------------------------ auxiliary calls ----------- */
+
+/* Event-queue driver (the single queue of Sec. 4.1: worker results and global models are processed
+ * in arrival order; Appendix A: the trace is replayed in its recorded order). */
+enum { HALOS_EV_ARRIVE = 0, HALOS_EV_GPS_RECV = 1, HALOS_EV_PULL = 2 };
+
+typedef struct halos_event {
+    uint8_t kind;      /* HALOS_EV_* */
+    uint8_t lps;
+    uint16_t worker;   /* ARRIVE only */
+    uint32_t pad;
+    int64_t time_ns;   /* informational */
+} halos_event;
+
+typedef struct halos_event_log {
+    uint32_t index;            /* position in the trace */
+    uint8_t kind, lps;
+    uint16_t worker;
+    uint64_t t, t_last;        /* LPS counters after the event */
+    uint64_t gps_iter;         /* GPS iteration i after the event */
+    uint64_t worker_staleness; /* ARRIVE: LPS updates applied since this worker was scheduled */
+    uint64_t gps_lag;          /* PULL: GPS iterations since the merged Theta_i was produced */
+    uint8_t pushed;            /* ARRIVE: this arrival completed a window of K and pushed */
+    uint8_t fused;             /* the event ran inside a fused launch */
+    uint8_t pad[6];
+} halos_event_log;
+
+/* Called by halos_replay before each ARRIVE to obtain the worker's result theta_{t,H}: fill exactly
+ * one of *flat_dev / *ptrs_host (same meaning as in halos_worker_delta).  `round` counts this
+ * worker's arrivals from 0.  Any work the producer enqueues must go to the context's stream.
+ * Return 0, or nonzero to abort the replay. */
+typedef int (*halos_producer_fn)(void* user, uint32_t event_index, uint32_t worker, uint64_t round,
+                                 const void** flat_dev, const void* const** ptrs_host);
+
+/* Replays events[0..n) in order: ARRIVE = worker_delta + lps_apply (+ lps_push when the window of
+ * K closes, fused into the same launch), GPS_RECV = gps_merge, PULL = lps_pull.  log_host (may be
+ * NULL) receives one record per event.  Stops at the first failing event: returns its status and
+ * writes its index to *failed_at (may be NULL); events before it stay applied. */
+int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
+                 void* user, halos_event_log* log_host, uint32_t* failed_at);
+
+/* Read-only device pointer to a state buffer (for inspection; valid until halos_destroy).
+ * *numel = P.  Element type fp32, or worker_dtype for HALOS_BUF_THETA0. */
+int halos_peek(halos_ctx* ctx, uint32_t which, uint32_t index, const void** ptr_dev, uint64_t* numel);
+
+/* Copies elements [offset, offset+count) of a state buffer to host memory, in stream order, and
+ * waits for the copy. */
+int halos_read(halos_ctx* ctx, uint32_t which, uint32_t index, uint64_t offset, uint64_t count,
+               void* dst_host);
+
+/* counters_host[5] = { t, t_last, phase, t at the last push, GPS iteration i } for one LPS. */
+int halos_counters(halos_ctx* ctx, uint32_t lps, uint64_t* counters_host);
+
+/* info_host[3] = { arrivals seen from the worker, LPS counter t when it was last scheduled, pending } */
+int halos_worker_info(halos_ctx* ctx, uint32_t worker, uint64_t* info_host);
+
+/* Per-tensor squared norms (needs HALOS_FLAG_STATS): what = 0: sum delta^2 of the last
+ * halos_lps_apply of this LPS; what = 1: sum Delta^2 of its last halos_lps_push.  Waits for the
+ * stream.  out_host: [n_tensors] doubles. */
+int halos_stats(halos_ctx* ctx, uint32_t what, uint32_t lps, double* out_host);
+
+/* Number of parameters P, tensors, scheduler chunks, and kernels launched so far. */
+int halos_info(halos_ctx* ctx, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunks, uint64_t* launches);
+
+/* Per-kernel device timing.  While enabled, every update kernel is bracketed by CUDA events on the
+ * context's stream; halos_timing_read waits for the stream and returns, for one kernel kind, how
+ * many launches were timed since halos_timing_enable(ctx, 1) and their summed duration. */
+enum {
+    HALOS_K_ARRIVE = 0,       /* delta + LPS momentum update + schedule copy */
+    HALOS_K_ARRIVE_PUSH = 1,  /* the same, plus Delta formed in the same pass */
+    HALOS_K_PUSH = 2,
+    HALOS_K_GPS = 3,          /* global momentum update + Theta_i snapshot */
+    HALOS_K_PULL = 4,         /* merge + anchor reset */
+    HALOS_K_COUNT = 5
+};
+int halos_timing_enable(halos_ctx* ctx, int on);
+int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double* total_ms);
+
+const char* halos_strerror(int status);
+/* Text of the last error on this context (or of the last failed halos_create when ctx is NULL). */
+const char* halos_last_error(halos_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HALOS_H */

@@ -27,7 +27,7 @@ _SOURCES = [_HERE / "halos_oracle_c.cpp", _HERE / "halos_oracle.hpp"]
 
 F32, BF16 = 0, 1
 IDLE, PUSHED, ANSWERED = 0, 1, 2
-_WHICH = {"Theta": 0, "Mg": 1, "th": 2, "ml": 3, "anchor": 4, "outbox": 5, "inbox": 6, "th0": 7}
+_WHICH = {"Theta": 0, "Mg": 1, "th": 2, "ml": 3, "anchor": 4, "outbox": 5, "inbox": 6, "th0": 7, "delta": 8}
 
 
 def build(force: bool = False) -> Path:
@@ -153,7 +153,7 @@ class HalosOracle:
 
     # --- state ----------------------------------------------------------------------------
     def buffer(self, which: str, idx: int = 0) -> np.ndarray:
-        """numpy view (no copy) of one state buffer: Theta, Mg, th, ml, anchor, outbox, inbox, th0."""
+        """numpy view (no copy) of one state buffer: Theta, Mg, th, ml, anchor, outbox, inbox, th0, delta."""
         p = self._lib.halos_oracle_buffer(self._h, _WHICH[which], int(idx))
         if not p:
             raise IndexError(f"{which}[{idx}]")
@@ -163,6 +163,12 @@ class HalosOracle:
             ct, dt = (ctypes.c_float, np.float32) if self.dtype == np.float32 else (ctypes.c_double, np.float64)
         arr = np.ctypeslib.as_array(ctypes.cast(p, ctypes.POINTER(ct)), shape=(self.P,))
         return arr.view(dt)
+
+    def sq_norms(self, which: str, idx: int, offsets) -> np.ndarray:
+        """Per-tensor sum of squares of a buffer, accumulated in fp64 (tensor k = [offsets[k], offsets[k+1]))."""
+        x = self.buffer(which, idx).astype(np.float64)
+        off = np.asarray(offsets, dtype=np.int64)
+        return np.array([float(np.dot(x[a:b], x[a:b])) for a, b in zip(off[:-1], off[1:])])
 
     def counters(self, lps: int) -> dict:
         out = (ctypes.c_uint64 * 5)()

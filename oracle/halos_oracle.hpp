@@ -74,6 +74,7 @@ struct Config {
 template <class T>
 struct Lps {
     std::vector<T> th, ml, anchor, outbox, inbox;
+    std::vector<T> last_delta;  // the worker displacement applied by the most recent arrival (observability)
     uint64_t t = 0, t_last = 0, t_push = 0;
     int phase = IDLE;
 };
@@ -107,6 +108,7 @@ public:
             s.ml.assign(P, T(0));
             s.outbox.assign(P, T(0));
             s.inbox.assign(P, T(0));
+            s.last_delta.assign(P, T(0));
         }
         worker_round.assign(c.n_workers, 0);
         worker_sched_t.assign(c.n_workers, 0);
@@ -143,6 +145,7 @@ public:
             float* s0 = th0_f32[w].data();
             for (uint64_t j = 0; j < P; ++j) {
                 T d = (T)h[j] - (T)s0[j];                  // line 25: delta = theta_{t,H} - theta_{t,0}
+                s.last_delta[j] = d;
                 model_update(s.th[j], s.ml[j], d, eta, beta, omb);   // line 11
                 s0[j] = (float)s.th[j];                    // line 12: schedule the worker theta_t
             }
@@ -151,6 +154,7 @@ public:
             uint16_t* s0 = th0_bf16[w].data();
             for (uint64_t j = 0; j < P; ++j) {
                 T d = (T)bf16_to_f32(h[j]) - (T)bf16_to_f32(s0[j]);
+                s.last_delta[j] = d;
                 model_update(s.th[j], s.ml[j], d, eta, beta, omb);
                 s0[j] = f32_to_bf16_rne((float)s.th[j]);
             }

@@ -30,8 +30,8 @@ int guarded(Handle* h, F&& fn) {
 
 extern "C" {
 
-// which: 0 Theta, 1 Mg, 2 th[l], 3 ml[l], 4 anchor[l], 5 outbox[l], 6 inbox[l], 7 th0[w]
-enum { B_THETA = 0, B_MG, B_TH, B_ML, B_ANCHOR, B_OUTBOX, B_INBOX, B_TH0 };
+// which: 0 Theta, 1 Mg, 2 th[l], 3 ml[l], 4 anchor[l], 5 outbox[l], 6 inbox[l], 7 th0[w], 8 last delta[l]
+enum { B_THETA = 0, B_MG, B_TH, B_ML, B_ANCHOR, B_OUTBOX, B_INBOX, B_TH0, B_DELTA };
 
 void* halos_oracle_create(int use_double, uint64_t P, uint32_t n_lps, uint32_t n_workers,
                           const uint32_t* worker_lps, double eta_l, double beta_l, double eta_g,
@@ -107,6 +107,7 @@ void* halos_oracle_buffer(void* hv, int which, uint32_t idx) {
             case B_ANCHOR: return idx < o->lps.size() ? o->lps[idx].anchor.data() : nullptr;
             case B_OUTBOX: return idx < o->lps.size() ? o->lps[idx].outbox.data() : nullptr;
             case B_INBOX: return idx < o->lps.size() ? o->lps[idx].inbox.data() : nullptr;
+            case B_DELTA: return idx < o->lps.size() ? o->lps[idx].last_delta.data() : nullptr;
             case B_TH0:
                 if (idx >= o->cfg.n_workers) return nullptr;
                 return o->cfg.worker_dtype == W_F32 ? (void*)o->th0_f32[idx].data()

@@ -1,0 +1,745 @@
+// Host side of the HALoS server-path library: context, state machine of Algorithm 1, the
+// multi-tensor chunk table, kernel launches, and the C ABI declared in include/halos.h.
+#include "halos.h"
+#include "halos_kernels.cuh"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace halos;
+
+namespace {
+
+constexpr uint32_t kDefaultChunkElems = 8192;
+constexpr int kUnroll = 4;
+constexpr bool kStream = true;
+constexpr int kStageSlots = 2;
+
+thread_local std::string g_create_error;
+
+struct LpsState {
+    float *th = nullptr, *ml = nullptr, *anchor = nullptr, *outbox = nullptr, *inbox = nullptr;
+    uint64_t t = 0, t_last = 0, t_push = 0;
+    uint64_t inbox_iter = 0;  // GPS iteration that produced the inbox content
+    int phase = HALOS_IDLE;
+};
+
+enum { PEND_NONE = 0, PEND_FLAT = 1, PEND_PTRS = 2, PEND_STAGED = 3 };
+
+struct WorkerState {
+    void* th0 = nullptr;
+    uint32_t lps = 0;
+    int pending = PEND_NONE;
+    const void* flat = nullptr;
+    int slot = -1;
+    uint64_t round = 0;    // arrivals applied so far
+    uint64_t sched_t = 0;  // LPS counter when last scheduled
+    cudaEvent_t table_copied = nullptr;  // guards reuse of the pinned pointer-table slot
+};
+
+struct TimedLaunch {
+    cudaEvent_t a, b;
+    int kind;
+};
+
+}  // namespace
+
+struct halos_ctx {
+    halos_config cfg;
+    uint64_t P = 0;
+    uint32_t wb = 4;  // bytes per worker-copy element
+    std::vector<uint64_t> tensor_numel, tensor_off;
+    std::vector<uint32_t> worker_lps;
+    std::vector<Chunk> chunks;
+    std::vector<uint32_t> tensor_chunk_begin;
+    cudaStream_t stream = nullptr;
+    cudaStream_t copy_stream = nullptr;
+
+    Chunk* d_chunks = nullptr;
+    unsigned long long* d_tensor_off = nullptr;
+    uint32_t* d_tensor_chunk_begin = nullptr;
+    const void** d_ptr_tables = nullptr;  // [n_workers][n_tensors]
+    const void** h_ptr_tables = nullptr;  // pinned mirror
+    double *d_partial_delta = nullptr, *d_partial_Delta = nullptr;
+    double* d_stats = nullptr;  // [2][n_lps][n_tensors]
+
+    float *Theta = nullptr, *Mg = nullptr;
+    uint64_t gps_iter = 0;
+    std::vector<LpsState> lps;
+    std::vector<WorkerState> workers;
+
+    void* stage[kStageSlots] = {nullptr, nullptr};
+    cudaEvent_t stage_ready[kStageSlots] = {nullptr, nullptr};
+    cudaEvent_t stage_free[kStageSlots] = {nullptr, nullptr};
+    int stage_owner[kStageSlots] = {-1, -1};
+    int stage_next = 0;
+
+    std::vector<void*> owned;  // device allocations made through the allocator
+    uint64_t launches = 0;
+    bool timing = false;
+    std::vector<TimedLaunch> timed;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
+    std::string err;
+};
+
+namespace {
+
+int fail(halos_ctx* c, int status, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (c) c->err = buf;
+    else g_create_error = buf;
+    return status;
+}
+
+#define CU(c, call)                                                                                   \
+    do {                                                                                              \
+        cudaError_t e_ = (call);                                                                      \
+        if (e_ != cudaSuccess) return fail((c), HALOS_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+void* dev_alloc(halos_ctx* c, size_t bytes) {
+    if (bytes == 0) bytes = 256;
+    void* p = nullptr;
+    if (c->cfg.alloc) {
+        p = c->cfg.alloc(bytes, c->cfg.alloc_user);
+    } else if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        p = nullptr;
+    }
+    if (p) c->owned.push_back(p);
+    return p;
+}
+
+void release(halos_ctx* c) {
+    cudaStreamSynchronize(c->stream);
+    if (c->copy_stream) {
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamDestroy(c->copy_stream);
+    }
+    for (void* p : c->owned) {
+        if (c->cfg.free_ && c->cfg.alloc) c->cfg.free_(p, c->cfg.alloc_user);
+        else cudaFree(p);
+    }
+    c->owned.clear();
+    if (c->h_ptr_tables) cudaFreeHost((void*)c->h_ptr_tables);
+    for (auto& w : c->workers)
+        if (w.table_copied) cudaEventDestroy(w.table_copied);
+    for (int s = 0; s < kStageSlots; ++s) {
+        if (c->stage_ready[s]) cudaEventDestroy(c->stage_ready[s]);
+        if (c->stage_free[s]) cudaEventDestroy(c->stage_free[s]);
+    }
+    for (auto& t : c->timed) {
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    for (auto& e : c->event_pool) {
+        cudaEventDestroy(e.first);
+        cudaEventDestroy(e.second);
+    }
+    (void)cudaGetLastError();
+}
+
+// The chunk table: each tensor is cut into an unaligned head (0-3 elements, so that everything
+// after it starts on a 16-byte boundary of the packed fp32 state), full chunks, and a tail.
+void build_chunks(halos_ctx* c, uint32_t chunk_elems) {
+    c->chunks.clear();
+    c->tensor_chunk_begin.assign(c->tensor_numel.size() + 1, 0);
+    for (size_t k = 0; k < c->tensor_numel.size(); ++k) {
+        c->tensor_chunk_begin[k] = (uint32_t)c->chunks.size();
+        uint64_t pos = c->tensor_off[k], end = c->tensor_off[k] + c->tensor_numel[k];
+        uint64_t head = (4 - (pos & 3)) & 3;
+        if (head && pos < end) {
+            uint64_t n = head < end - pos ? head : end - pos;
+            c->chunks.push_back(Chunk{pos, (uint32_t)n, (uint32_t)k});
+            pos += n;
+        }
+        while (pos < end) {
+            uint64_t n = end - pos < chunk_elems ? end - pos : chunk_elems;
+            c->chunks.push_back(Chunk{pos, (uint32_t)n, (uint32_t)k});
+            pos += n;
+        }
+    }
+    c->tensor_chunk_begin[c->tensor_numel.size()] = (uint32_t)c->chunks.size();
+}
+
+struct Timer {
+    halos_ctx* c;
+    cudaEvent_t a = nullptr, b = nullptr;
+    int kind;
+    Timer(halos_ctx* c_, int kind_) : c(c_), kind(kind_) {
+        if (!c->timing) return;
+        if (!c->event_pool.empty()) {
+            a = c->event_pool.back().first;
+            b = c->event_pool.back().second;
+            c->event_pool.pop_back();
+        } else if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+            a = b = nullptr;
+            (void)cudaGetLastError();
+            return;
+        }
+        cudaEventRecord(a, c->stream);
+    }
+    void stop() {
+        if (!a) return;
+        cudaEventRecord(b, c->stream);
+        c->timed.push_back(TimedLaunch{a, b, kind});
+    }
+};
+
+template <class W>
+int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
+    ArriveArgs<W> a;
+    a.h_flat = (const W*)flat;
+    a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)widx * c->tensor_numel.size());
+    a.tensor_off = c->d_tensor_off;
+    a.th0 = (W*)w.th0;
+    a.th = s.th;
+    a.ml = s.ml;
+    a.anchor = s.anchor;
+    a.outbox = s.outbox;
+    a.partial_delta = c->d_partial_delta;
+    a.partial_Delta = c->d_partial_Delta;
+    a.eta = c->cfg.eta_l;
+    a.beta = c->cfg.beta_l;
+    a.omb = 1.0f - c->cfg.beta_l;
+    const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    if (grid.x == 0) return HALOS_OK;
+    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+    if (push) {
+        if (stats) arrive_kernel<W, true, true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_kernel<W, true, false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    } else {
+        if (stats) arrive_kernel<W, false, true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_kernel<W, false, false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    }
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+
+int finalize_stats(halos_ctx* c, uint32_t what, uint32_t lps) {
+    const uint32_t nt = (uint32_t)c->tensor_numel.size();
+    double* out = c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt;
+    const double* partial = what == 0 ? c->d_partial_delta : c->d_partial_Delta;
+    stats_finalize_kernel<<<nt, 32, 0, c->stream>>>(partial, c->d_tensor_chunk_begin, out, nt);
+    c->launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+
+// lps_apply with an optional fused push; shared by the C entry point and the replay driver.
+int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int* push_due) {
+    if (lps >= c->cfg.n_lps || worker >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "lps/worker out of range");
+    WorkerState& w = c->workers[worker];
+    if (w.lps != lps) return fail(c, HALOS_ERR_INVALID_ARG, "worker %u does not belong to LPS %u", worker, lps);
+    if (w.pending == PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u has no pending result", worker);
+    LpsState& s = c->lps[lps];
+    const bool due = (s.t + 1 - s.t_last == c->cfg.K);
+    const bool push = fuse_push && due;
+    if (push && s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u: push due while a round trip is in flight", lps);
+    CU(c, cudaSetDevice(c->cfg.device));
+    const void* flat = nullptr;
+    if (w.pending == PEND_FLAT) flat = w.flat;
+    if (w.pending == PEND_STAGED) {
+        flat = c->stage[w.slot];
+        CU(c, cudaStreamWaitEvent(c->stream, c->stage_ready[w.slot], 0));
+    }
+    int rc = c->wb == 4 ? launch_arrive<float>(c, s, w, worker, push, flat)
+                        : launch_arrive<uint16_t>(c, s, w, worker, push, flat);
+    if (rc != HALOS_OK) return rc;
+    if (w.pending == PEND_STAGED) {
+        CU(c, cudaEventRecord(c->stage_free[w.slot], c->stream));
+        c->stage_owner[w.slot] = -1;
+    }
+    if (c->cfg.flags & HALOS_FLAG_STATS) {
+        if ((rc = finalize_stats(c, 0, lps)) != HALOS_OK) return rc;
+        if (push && (rc = finalize_stats(c, 1, lps)) != HALOS_OK) return rc;
+    }
+    w.pending = PEND_NONE;
+    w.flat = nullptr;
+    w.slot = -1;
+    w.round += 1;
+    s.t += 1;
+    w.sched_t = s.t;
+    if (push) {
+        s.phase = HALOS_PUSHED;
+        s.t_push = s.t;
+    }
+    if (push_due) *push_due = due ? 1 : 0;
+    return HALOS_OK;
+}
+
+}  // namespace
+
+// ====================================================================================== C ABI
+extern "C" {
+
+void halos_default_config(halos_config* cfg) {
+    if (!cfg) return;
+    std::memset(cfg, 0, sizeof *cfg);
+    cfg->struct_size = (uint32_t)sizeof(halos_config);
+    cfg->eta_l = 0.2f;
+    cfg->beta_l = 0.9f;
+    cfg->eta_g = 0.15f;
+    cfg->beta_g = 0.5f;
+    cfg->alpha = 0.25f;
+    cfg->K = 32;
+    cfg->worker_dtype = HALOS_F32;
+}
+
+int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx** out) {
+    if (!cfg || !out || !theta_init_dev) return fail(nullptr, HALOS_ERR_INVALID_ARG, "null argument");
+    if (cfg->struct_size != sizeof(halos_config)) return fail(nullptr, HALOS_ERR_INVALID_ARG, "struct_size mismatch");
+    if (cfg->n_lps == 0 || cfg->n_workers == 0 || cfg->n_tensors == 0 || !cfg->worker_lps || !cfg->tensor_numel)
+        return fail(nullptr, HALOS_ERR_INVALID_ARG, "empty configuration");
+    if (cfg->n_lps > 255 || cfg->n_workers > 65535) return fail(nullptr, HALOS_ERR_INVALID_ARG, "too many servers or workers");
+    if (cfg->K == 0) return fail(nullptr, HALOS_ERR_INVALID_ARG, "K must be positive");
+    if (cfg->worker_dtype != HALOS_F32 && cfg->worker_dtype != HALOS_BF16)
+        return fail(nullptr, HALOS_ERR_INVALID_ARG, "unknown worker_dtype");
+    if ((cfg->alloc == nullptr) != (cfg->free_ == nullptr)) return fail(nullptr, HALOS_ERR_INVALID_ARG, "alloc and free_ go together");
+    for (uint32_t w = 0; w < cfg->n_workers; ++w)
+        if (cfg->worker_lps[w] >= cfg->n_lps) return fail(nullptr, HALOS_ERR_INVALID_ARG, "worker_lps[%u] out of range", w);
+    uint32_t chunk_elems = cfg->chunk_elems ? cfg->chunk_elems : kDefaultChunkElems;
+    if (chunk_elems % 4 != 0 || chunk_elems < 4) return fail(nullptr, HALOS_ERR_INVALID_ARG, "chunk_elems must be a positive multiple of 4");
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+        (void)cudaGetLastError();
+        return fail(nullptr, HALOS_ERR_CUDA, "no CUDA device: this library has no CPU path");
+    }
+    if (cfg->device < 0 || cfg->device >= ndev) return fail(nullptr, HALOS_ERR_INVALID_ARG, "device ordinal out of range");
+
+    halos_ctx* c = new (std::nothrow) halos_ctx();
+    if (!c) return fail(nullptr, HALOS_ERR_OOM, "host allocation failed");
+    c->cfg = *cfg;
+    c->cfg.worker_lps = nullptr;
+    c->cfg.tensor_numel = nullptr;
+    c->stream = (cudaStream_t)cfg->stream;
+    c->wb = cfg->worker_dtype == HALOS_F32 ? 4 : 2;
+    c->worker_lps.assign(cfg->worker_lps, cfg->worker_lps + cfg->n_workers);
+    c->tensor_numel.assign(cfg->tensor_numel, cfg->tensor_numel + cfg->n_tensors);
+    c->tensor_off.resize(cfg->n_tensors + 1);
+    c->tensor_off[0] = 0;
+    for (uint32_t k = 0; k < cfg->n_tensors; ++k) c->tensor_off[k + 1] = c->tensor_off[k] + c->tensor_numel[k];
+    c->P = c->tensor_off[cfg->n_tensors];
+    if (c->P == 0) {
+        delete c;
+        return fail(nullptr, HALOS_ERR_INVALID_ARG, "P = 0");
+    }
+    build_chunks(c, chunk_elems);
+
+    auto bail = [&](int status, const char* what) {
+        std::string msg = c->err.empty() ? what : c->err;
+        release(c);
+        delete c;
+        return fail(nullptr, status, "%s", msg.c_str());
+    };
+#define CUC(call)                                                                  \
+    do {                                                                           \
+        cudaError_t e_ = (call);                                                   \
+        if (e_ != cudaSuccess) {                                                   \
+            c->err = std::string(#call) + ": " + cudaGetErrorString(e_);           \
+            return bail(HALOS_ERR_CUDA, "cuda");                                   \
+        }                                                                          \
+    } while (0)
+
+    CUC(cudaSetDevice(cfg->device));
+    const size_t P = c->P, nt = cfg->n_tensors, nc = c->chunks.size();
+    auto A = [&](size_t bytes) { return dev_alloc(c, bytes); };
+    bool ok = true;
+    ok &= (c->d_chunks = (Chunk*)A(nc * sizeof(Chunk))) != nullptr;
+    ok &= (c->d_tensor_off = (unsigned long long*)A((nt + 1) * 8)) != nullptr;
+    ok &= (c->d_tensor_chunk_begin = (uint32_t*)A((nt + 1) * 4)) != nullptr;
+    ok &= (c->d_ptr_tables = (const void**)A((size_t)cfg->n_workers * nt * 8)) != nullptr;
+    if (cfg->flags & HALOS_FLAG_STATS) {
+        ok &= (c->d_partial_delta = (double*)A(nc * 8)) != nullptr;
+        ok &= (c->d_partial_Delta = (double*)A(nc * 8)) != nullptr;
+        ok &= (c->d_stats = (double*)A((size_t)2 * cfg->n_lps * nt * 8)) != nullptr;
+    }
+    ok &= (c->Theta = (float*)A(P * 4)) != nullptr;
+    ok &= (c->Mg = (float*)A(P * 4)) != nullptr;
+    c->lps.resize(cfg->n_lps);
+    for (auto& s : c->lps) {
+        if (!ok) break;
+        ok &= (s.th = (float*)A(P * 4)) != nullptr;
+        ok &= (s.ml = (float*)A(P * 4)) != nullptr;
+        ok &= (s.anchor = (float*)A(P * 4)) != nullptr;
+        ok &= (s.outbox = (float*)A(P * 4)) != nullptr;
+        ok &= (s.inbox = (float*)A(P * 4)) != nullptr;
+    }
+    c->workers.resize(cfg->n_workers);
+    for (uint32_t w = 0; w < cfg->n_workers && ok; ++w) {
+        c->workers[w].lps = c->worker_lps[w];
+        ok &= (c->workers[w].th0 = A(P * c->wb)) != nullptr;
+    }
+    if (!ok) return bail(HALOS_ERR_OOM, "device allocation failed");
+    for (void* p : c->owned)
+        if (reinterpret_cast<uintptr_t>(p) & 255) return bail(HALOS_ERR_INVALID_ARG, "allocator returned a pointer not aligned to 256 bytes");
+
+    CUC(cudaHostAlloc((void**)&c->h_ptr_tables, (size_t)cfg->n_workers * nt * 8, cudaHostAllocDefault));
+    for (auto& w : c->workers) CUC(cudaEventCreateWithFlags(&w.table_copied, cudaEventDisableTiming));
+    CUC(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    for (int s = 0; s < kStageSlots; ++s) {
+        CUC(cudaEventCreateWithFlags(&c->stage_ready[s], cudaEventDisableTiming));
+        CUC(cudaEventCreateWithFlags(&c->stage_free[s], cudaEventDisableTiming));
+    }
+
+    cudaStream_t st = c->stream;
+    CUC(cudaMemcpyAsync(c->d_chunks, c->chunks.data(), nc * sizeof(Chunk), cudaMemcpyHostToDevice, st));
+    CUC(cudaMemcpyAsync(c->d_tensor_off, c->tensor_off.data(), (nt + 1) * 8, cudaMemcpyHostToDevice, st));
+    CUC(cudaMemcpyAsync(c->d_tensor_chunk_begin, c->tensor_chunk_begin.data(), (nt + 1) * 4, cudaMemcpyHostToDevice, st));
+    if (c->d_stats) CUC(cudaMemsetAsync(c->d_stats, 0, (size_t)2 * cfg->n_lps * nt * 8, st));
+    // Alg. 1 lines 6-7
+    CUC(cudaMemcpyAsync(c->Theta, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
+    CUC(cudaMemsetAsync(c->Mg, 0, P * 4, st));
+    for (auto& s : c->lps) {
+        CUC(cudaMemcpyAsync(s.th, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
+        CUC(cudaMemcpyAsync(s.anchor, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
+        CUC(cudaMemsetAsync(s.ml, 0, P * 4, st));
+        CUC(cudaMemsetAsync(s.outbox, 0, P * 4, st));
+        CUC(cudaMemsetAsync(s.inbox, 0, P * 4, st));
+    }
+    for (auto& w : c->workers) {
+        if (c->wb == 4) {
+            CUC(cudaMemcpyAsync(w.th0, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
+        } else {
+            cast_bf16_kernel<<<1184, 256, 0, st>>>(theta_init_dev, (uint16_t*)w.th0, (unsigned long long)P);
+            CUC(cudaGetLastError());
+        }
+    }
+    CUC(cudaStreamSynchronize(st));
+#undef CUC
+    *out = c;
+    return HALOS_OK;
+}
+
+int halos_destroy(halos_ctx* c) {
+    if (!c) return HALOS_OK;
+    cudaSetDevice(c->cfg.device);
+    release(c);
+    delete c;
+    return HALOS_OK;
+}
+
+int halos_worker_delta(halos_ctx* c, uint32_t worker, const void* flat, const void* const* ptrs) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (worker >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "worker out of range");
+    if ((flat == nullptr) == (ptrs == nullptr)) return fail(c, HALOS_ERR_INVALID_ARG, "give exactly one of flat / pointer table");
+    WorkerState& w = c->workers[worker];
+    if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u already has a pending result", worker);
+    if (flat) {
+        if (reinterpret_cast<uintptr_t>(flat) % c->wb) return fail(c, HALOS_ERR_INVALID_ARG, "thetaH not aligned to its element size");
+        w.flat = flat;
+        w.pending = PEND_FLAT;
+        return HALOS_OK;
+    }
+    const size_t nt = c->tensor_numel.size();
+    for (size_t k = 0; k < nt; ++k) {
+        if (!ptrs[k] && c->tensor_numel[k]) return fail(c, HALOS_ERR_INVALID_ARG, "null pointer for tensor %zu", k);
+        if (reinterpret_cast<uintptr_t>(ptrs[k]) % c->wb) return fail(c, HALOS_ERR_INVALID_ARG, "tensor %zu not aligned to its element size", k);
+    }
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaEventSynchronize(w.table_copied));  // the previous upload from this pinned slot has left the host
+    const void** slot = c->h_ptr_tables + (size_t)worker * nt;
+    std::memcpy(slot, ptrs, nt * 8);
+    CU(c, cudaMemcpyAsync(c->d_ptr_tables + (size_t)worker * nt, slot, nt * 8, cudaMemcpyHostToDevice, c->stream));
+    CU(c, cudaEventRecord(w.table_copied, c->stream));
+    w.pending = PEND_PTRS;
+    return HALOS_OK;
+}
+
+int halos_worker_delta_host(halos_ctx* c, uint32_t worker, const void* host) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (worker >= c->cfg.n_workers || !host) return fail(c, HALOS_ERR_INVALID_ARG, "bad worker or null pointer");
+    WorkerState& w = c->workers[worker];
+    if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u already has a pending result", worker);
+    int slot = -1;
+    for (int k = 0; k < kStageSlots; ++k) {
+        int s = (c->stage_next + k) % kStageSlots;
+        if (c->stage_owner[s] < 0) {
+            slot = s;
+            break;
+        }
+    }
+    if (slot < 0) return fail(c, HALOS_ERR_BAD_STATE, "all %d staging buffers hold results that were not applied yet", kStageSlots);
+    CU(c, cudaSetDevice(c->cfg.device));
+    if (!c->stage[slot]) {
+        c->stage[slot] = dev_alloc(c, c->P * c->wb);
+        if (!c->stage[slot]) return fail(c, HALOS_ERR_OOM, "staging buffer allocation failed");
+    }
+    // The copy runs on the context's own copy stream so that it overlaps the update kernels of
+    // earlier events; stage_free orders it after the kernel that last read this slot.
+    CU(c, cudaStreamWaitEvent(c->copy_stream, c->stage_free[slot], 0));
+    CU(c, cudaMemcpyAsync(c->stage[slot], host, c->P * c->wb, cudaMemcpyHostToDevice, c->copy_stream));
+    CU(c, cudaEventRecord(c->stage_ready[slot], c->copy_stream));
+    c->stage_owner[slot] = (int)worker;
+    c->stage_next = (slot + 1) % kStageSlots;
+    w.slot = slot;
+    w.pending = PEND_STAGED;
+    return HALOS_OK;
+}
+
+int halos_lps_apply(halos_ctx* c, uint32_t lps, uint32_t worker, int* push_due) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    return apply_impl(c, lps, worker, false, push_due);
+}
+
+int halos_lps_push(halos_ctx* c, uint32_t lps) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    LpsState& s = c->lps[lps];
+    if (s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u already has a round trip in flight", lps);
+    CU(c, cudaSetDevice(c->cfg.device));
+    PushArgs a{s.th, s.anchor, s.outbox, c->d_partial_Delta};
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
+    Timer tm(c, HALOS_K_PUSH);
+    if (stats) push_kernel<true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    else push_kernel<false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    if (stats) {
+        int rc = finalize_stats(c, 1, lps);
+        if (rc != HALOS_OK) return rc;
+    }
+    s.phase = HALOS_PUSHED;
+    s.t_push = s.t;
+    return HALOS_OK;
+}
+
+int halos_gps_merge(halos_ctx* c, uint32_t lps) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    LpsState& s = c->lps[lps];
+    if (s.phase != HALOS_PUSHED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Delta in flight", lps);
+    CU(c, cudaSetDevice(c->cfg.device));
+    GpsArgs a{s.outbox, c->Theta, c->Mg, s.inbox, c->cfg.eta_g, c->cfg.beta_g, 1.0f - c->cfg.beta_g};
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    Timer tm(c, HALOS_K_GPS);
+    gps_kernel<kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    c->gps_iter += 1;
+    s.inbox_iter = c->gps_iter;
+    s.phase = HALOS_ANSWERED;
+    return HALOS_OK;
+}
+
+int halos_lps_pull(halos_ctx* c, uint32_t lps) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    LpsState& s = c->lps[lps];
+    if (s.phase != HALOS_ANSWERED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Theta_i to merge", lps);
+    CU(c, cudaSetDevice(c->cfg.device));
+    PullArgs a{s.th, s.inbox, s.anchor, c->cfg.alpha, 1.0f - c->cfg.alpha};
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    Timer tm(c, HALOS_K_PULL);
+    pull_kernel<kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    s.t_last = s.t;
+    s.phase = HALOS_IDLE;
+    return HALOS_OK;
+}
+
+// ------------------------------------------------------------------------------ event-queue driver
+int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
+                 halos_event_log* log, uint32_t* failed_at) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (n && !ev) return fail(c, HALOS_ERR_INVALID_ARG, "null event array");
+    for (uint32_t k = 0; k < n; ++k) {
+        const halos_event& e = ev[k];
+        int rc = HALOS_OK;
+        halos_event_log rec;
+        std::memset(&rec, 0, sizeof rec);
+        rec.index = k;
+        rec.kind = e.kind;
+        rec.lps = e.lps;
+        rec.worker = e.worker;
+        if (e.lps >= c->cfg.n_lps) rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: lps out of range", k);
+        else if (e.kind == HALOS_EV_ARRIVE) {
+            if (e.worker >= c->cfg.n_workers) rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: worker out of range", k);
+            else if (!producer) rc = fail(c, HALOS_ERR_INVALID_ARG, "ARRIVE events need a producer");
+            else {
+                WorkerState& w = c->workers[e.worker];
+                const void* flat = nullptr;
+                const void* const* ptrs = nullptr;
+                if (w.pending == PEND_NONE) {
+                    if (producer(user, k, e.worker, w.round, &flat, &ptrs) != 0)
+                        rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: producer failed", k);
+                    else rc = halos_worker_delta(c, e.worker, flat, ptrs);
+                }
+                if (rc == HALOS_OK) {
+                    rec.worker_staleness = c->lps[e.lps].t - w.sched_t;
+                    int due = 0;
+                    rc = apply_impl(c, e.lps, e.worker, true, &due);
+                    rec.pushed = (uint8_t)due;
+                    rec.fused = (uint8_t)due;
+                }
+            }
+        } else if (e.kind == HALOS_EV_GPS_RECV) {
+            rc = halos_gps_merge(c, e.lps);
+        } else if (e.kind == HALOS_EV_PULL) {
+            if (c->lps[e.lps].phase == HALOS_ANSWERED) rec.gps_lag = c->gps_iter - c->lps[e.lps].inbox_iter;
+            rc = halos_lps_pull(c, e.lps);
+        } else {
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: unknown kind %u", k, (unsigned)e.kind);
+        }
+        if (rc != HALOS_OK) {
+            if (failed_at) *failed_at = k;
+            return rc;
+        }
+        if (log) {
+            rec.t = c->lps[e.lps].t;
+            rec.t_last = c->lps[e.lps].t_last;
+            rec.gps_iter = c->gps_iter;
+            log[k] = rec;
+        }
+    }
+    return HALOS_OK;
+}
+
+// ------------------------------------------------------------------------------ inspection
+static int buffer_of(halos_ctx* c, uint32_t which, uint32_t index, const void** p, uint32_t* elem_bytes) {
+    *elem_bytes = 4;
+    switch (which) {
+        case HALOS_BUF_THETA_G: *p = c->Theta; return HALOS_OK;
+        case HALOS_BUF_M_G: *p = c->Mg; return HALOS_OK;
+        case HALOS_BUF_THETA_L: case HALOS_BUF_M_L: case HALOS_BUF_ANCHOR: case HALOS_BUF_OUTBOX: case HALOS_BUF_INBOX: {
+            if (index >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+            LpsState& s = c->lps[index];
+            *p = which == HALOS_BUF_THETA_L ? s.th : which == HALOS_BUF_M_L ? s.ml : which == HALOS_BUF_ANCHOR ? s.anchor
+                 : which == HALOS_BUF_OUTBOX ? s.outbox : s.inbox;
+            return HALOS_OK;
+        }
+        case HALOS_BUF_THETA0:
+            if (index >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "worker out of range");
+            *p = c->workers[index].th0;
+            *elem_bytes = c->wb;
+            return HALOS_OK;
+    }
+    return fail(c, HALOS_ERR_INVALID_ARG, "unknown buffer id %u", which);
+}
+
+int halos_peek(halos_ctx* c, uint32_t which, uint32_t index, const void** ptr_dev, uint64_t* numel) {
+    if (!c || !ptr_dev) return HALOS_ERR_INVALID_ARG;
+    const void* p;
+    uint32_t eb;
+    int rc = buffer_of(c, which, index, &p, &eb);
+    if (rc != HALOS_OK) return rc;
+    *ptr_dev = p;
+    if (numel) *numel = c->P;
+    return HALOS_OK;
+}
+
+int halos_read(halos_ctx* c, uint32_t which, uint32_t index, uint64_t offset, uint64_t count, void* dst) {
+    if (!c || (!dst && count)) return HALOS_ERR_INVALID_ARG;
+    const void* p;
+    uint32_t eb;
+    int rc = buffer_of(c, which, index, &p, &eb);
+    if (rc != HALOS_OK) return rc;
+    if (offset > c->P || count > c->P - offset) return fail(c, HALOS_ERR_INVALID_ARG, "range outside the buffer");
+    if (count == 0) return HALOS_OK;
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaMemcpyAsync(dst, (const char*)p + offset * eb, count * eb, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return HALOS_OK;
+}
+
+int halos_counters(halos_ctx* c, uint32_t lps, uint64_t* out) {
+    if (!c || !out) return HALOS_ERR_INVALID_ARG;
+    if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    const LpsState& s = c->lps[lps];
+    out[0] = s.t;
+    out[1] = s.t_last;
+    out[2] = (uint64_t)s.phase;
+    out[3] = s.t_push;
+    out[4] = c->gps_iter;
+    return HALOS_OK;
+}
+
+int halos_worker_info(halos_ctx* c, uint32_t worker, uint64_t* out) {
+    if (!c || !out) return HALOS_ERR_INVALID_ARG;
+    if (worker >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "worker out of range");
+    out[0] = c->workers[worker].round;
+    out[1] = c->workers[worker].sched_t;
+    out[2] = c->workers[worker].pending != PEND_NONE;
+    return HALOS_OK;
+}
+
+int halos_stats(halos_ctx* c, uint32_t what, uint32_t lps, double* out) {
+    if (!c || !out) return HALOS_ERR_INVALID_ARG;
+    if (!(c->cfg.flags & HALOS_FLAG_STATS)) return fail(c, HALOS_ERR_BAD_STATE, "context was created without HALOS_FLAG_STATS");
+    if (what > 1 || lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "bad statistic or lps");
+    const size_t nt = c->tensor_numel.size();
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaMemcpyAsync(out, c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt, nt * 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return HALOS_OK;
+}
+
+int halos_info(halos_ctx* c, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunks, uint64_t* launches) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (P) *P = c->P;
+    if (n_tensors) *n_tensors = (uint32_t)c->tensor_numel.size();
+    if (n_chunks) *n_chunks = (uint32_t)c->chunks.size();
+    if (launches) *launches = c->launches;
+    return HALOS_OK;
+}
+
+int halos_timing_enable(halos_ctx* c, int on) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->stream));
+    for (auto& t : c->timed) c->event_pool.emplace_back(t.a, t.b);
+    c->timed.clear();
+    c->timing = on != 0;
+    return HALOS_OK;
+}
+
+int halos_timing_read(halos_ctx* c, uint32_t kind, uint64_t* launches, double* total_ms) {
+    if (!c || kind >= HALOS_K_COUNT) return HALOS_ERR_INVALID_ARG;
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->stream));
+    uint64_t n = 0;
+    double ms = 0.0;
+    for (auto& t : c->timed) {
+        if (t.kind != (int)kind) continue;
+        float x = 0.f;
+        CU(c, cudaEventElapsedTime(&x, t.a, t.b));
+        ms += x;
+        n += 1;
+    }
+    if (launches) *launches = n;
+    if (total_ms) *total_ms = ms;
+    return HALOS_OK;
+}
+
+const char* halos_strerror(int status) {
+    switch (status) {
+        case HALOS_OK: return "ok";
+        case HALOS_ERR_INVALID_ARG: return "invalid argument";
+        case HALOS_ERR_BAD_STATE: return "call order violates the update rules";
+        case HALOS_ERR_OOM: return "out of memory";
+        case HALOS_ERR_CUDA: return "CUDA error";
+        case HALOS_ERR_UNSUPPORTED: return "unsupported";
+    }
+    return "unknown status";
+}
+
+const char* halos_last_error(halos_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

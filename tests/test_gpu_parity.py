@@ -1,0 +1,327 @@
+"""Parity of the CUDA library (called through the C ABI) with the CPU oracle on the same seeded
+traces and inputs.  Tolerances: max relative error 1e-6 after any single event, 1e-5 after a full
+trace (fp32); the arithmetic is mirrored operation by operation, so bit identity is expected and
+asserted wherever the whole state is compared."""
+from __future__ import annotations
+
+import struct
+import zlib
+from fractions import Fraction as Fr
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_04531_b200 import binding as hb
+from paper_2506_04531_b200.inputs import gen, layouts, trace as tr, workloads
+from parity_harness import FULL_TRACE_TOL, PER_EVENT_TOL, Lockstep, default_probes
+
+pytestmark = pytest.mark.gpu
+
+PAPER_HP = dict(eta_l=0.2, beta_l=0.9, eta_g=0.15, beta_g=0.5, alpha=0.25)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2506_04531_b200 import build
+    build.build()
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA input generator equals the numpy one bit for bit (they feed the two sides)
+# ---------------------------------------------------------------------------------------------
+def test_generators_agree():
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.decoder_layout("tiny", 2, 64, 300)
+    dg = DeviceGenerator(lay, 77)
+    init = dg.theta_init().cpu().numpy()
+    np.testing.assert_array_equal(init.view(np.uint32), gen.theta_init(lay, 77).view(np.uint32))
+    np.testing.assert_array_equal(dg.theta_init(1000, 5001).cpu().numpy(), init[1000:5001])
+    s0 = torch.from_numpy(init).cuda()
+    r = dg.worker_result(s0, 3, 9).cpu().numpy()
+    np.testing.assert_array_equal(r.view(np.uint32), gen.worker_result(init, lay, 77, 3, 9).view(np.uint32))
+    hb16 = gen.f32_to_bf16_bits(init)
+    s0b = torch.from_numpy(hb16.view(np.int16)).cuda()
+    rb = dg.worker_result(s0b, 3, 9, worker_dtype=gen.BF16).cpu().numpy().view(np.uint16)
+    np.testing.assert_array_equal(rb, gen.worker_result(hb16, lay, 77, 3, 9, worker_dtype=gen.BF16))
+
+
+# ---------------------------------------------------------------------------------------------
+# exact hand expansion on 8 parameters, straight against the golden values
+# ---------------------------------------------------------------------------------------------
+def test_hand_expansion_on_gpu():
+    golden = Path(__file__).parent / "golden" / "hand_expansion_p8.txt"
+    rows, bits = [], {}
+    for line in golden.read_text().splitlines():
+        parts = line.split()
+        if not parts or parts[0].startswith("#"):
+            continue
+        if parts[0] == "bits":
+            bits[parts[1]] = [int(x, 16) for x in parts[2:]]
+        else:
+            rows.append((int(parts[0]), parts[1], [float(Fr(x)) for x in parts[2:]]))
+    init = torch.tensor([(j - 4) / 8 for j in range(8)], dtype=torch.float32, device="cuda")
+    h = hb.Halos(init, [0, 0, 1], eta_l=0.5, beta_l=0.5, eta_g=0.5, beta_g=0.5, alpha=0.25, K=2)
+    which = {"th": hb.BUF_THETA_L, "ml": hb.BUF_M_L, "outbox": hb.BUF_OUTBOX}
+    rounds = [0, 0, 0]
+    for n, e in enumerate("A0 A2 A1 A0 G0 A2 G1 P0 A1 P1 A0 G0".split(), 1):
+        kind, i = e[0], int(e[1])
+        if kind == "A":
+            s0 = h.read(hb.BUF_THETA0, i)
+            noise = np.array([((3 * i + 5 * rounds[i] + 7 * j) % 9 - 4) / 16 for j in range(8)], np.float32)
+            rounds[i] += 1
+            thH = torch.from_numpy(s0 + noise).cuda()
+            h.worker_delta(i, thH)
+            if h.lps_apply(int(h.worker_lps[i]), i):
+                h.lps_push(int(h.worker_lps[i]))
+        elif kind == "G":
+            h.gps_merge(i)
+        else:
+            h.lps_pull(i)
+        for ev, name, vals in rows:
+            if ev != n:
+                continue
+            if name == "Theta":
+                got = h.read(hb.BUF_THETA_G)
+            elif name == "Mg":
+                got = h.read(hb.BUF_M_G)
+            else:
+                got = h.read(which[name[:-1]], int(name[-1]))
+            assert got.tolist() == vals, f"event {n} {name}"
+    as_bits = lambda a: [struct.unpack("<I", struct.pack("<f", float(x)))[0] for x in a]
+    assert as_bits(h.read(hb.BUF_THETA_G)) == bits["Theta"]
+    assert as_bits(h.read(hb.BUF_THETA_L, 0)) == bits["th0"]
+    assert as_bits(h.read(hb.BUF_THETA_L, 1)) == bits["th1"]
+    h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# tiny and ragged shapes, both worker dtypes, flat and pointer-table inputs, odd chunk sizes
+# ---------------------------------------------------------------------------------------------
+_SHAPES = {
+    "p1": [1], "p3": [3], "p4": [4], "p5": [5], "p8": [8], "p31": [31], "p4097": [4097],
+    "ragged": [7, 1, 1024, 3, 513, 2, 4096, 9, 1, 1, 777],
+    "ragged_big": [4099, 33, 20001, 5, 8192, 8191],
+    "with_empty": [16, 0, 5, 0, 64],
+}
+
+
+@pytest.mark.parametrize("shape", list(_SHAPES))
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+@pytest.mark.parametrize("mode", ["flat", "ptrs", "ptrs_misaligned"])
+def test_small_shapes_bit_exact(shape, wdt, mode):
+    lay = layouts.ragged_layout(shape, _SHAPES[shape])
+    worker_lps = [0, 0, 1, 1, 1]
+    events = tr.random_trace(worker_lps, 60, 3, seed=zlib.crc32(f"{shape}/{wdt}/{mode}".encode()) & 0xFFFF)
+    chunk = 1024 if shape in ("ragged_big", "p4097") else 0
+    ls = Lockstep(lay, worker_lps, dict(K=3, **PAPER_HP), wdt, seed=5, chunk_elems=chunk, input_mode=mode)
+    ls.run(events, check_every=1, full_check_every=20)
+    assert ls.bit_identical and ls.max_err == 0.0
+    ls.close()
+
+
+@pytest.mark.parametrize("chunk", [4, 64, 1024, 8192, 1 << 20])
+def test_chunk_size_invariance(chunk):
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 100000])
+    worker_lps = [0, 1]
+    events = tr.random_trace(worker_lps, 25, 2, seed=9)
+    ls = Lockstep(lay, worker_lps, dict(K=2, **PAPER_HP), gen.F32, seed=8, chunk_elems=chunk)
+    ls.run(events, check_every=5)
+    assert ls.bit_identical
+    info = ls.h.info()
+    assert info["P"] == lay.P and info["n_tensors"] == lay.n_tensors
+    ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# configuration 1 ("toy"): 1,048,576 parameters, 4 workers, 2 LPS, 200 arrivals, every event checked
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["toy", "toy_k4"])
+def test_toy_config_every_event(name):
+    wl = workloads.workload(name)
+    ls = Lockstep(wl.layout, wl.worker_lps, wl.hyper(), wl.worker_dtype, wl.seed)
+    ls.run(wl.trace(), check_every=1, full_check_every=50)
+    assert ls.bit_identical and ls.max_err <= PER_EVENT_TOL
+    # the trace exercised the whole hierarchy
+    kinds = [r["kind"] for r in ls.log]
+    assert kinds.count(tr.GPS_RECV) >= (20 if name == "toy_k4" else 4)
+    assert max(r.get("worker_staleness", 0) for r in ls.log) >= 1
+    ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the event-queue driver: same bits as the call-by-call sequence, and the same event log
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+def test_replay_driver_matches_calls_and_oracle_log(wdt):
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.decoder_layout("tiny", 2, 64, 300)
+    worker_lps = [0, 0, 1, 1]
+    hp = dict(K=4, **PAPER_HP)
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=[1.0, 2.5, 3.0, 1.7],
+                                            t_profiled_ms=1.0, n_arrivals=120, K=4))
+    ls = Lockstep(lay, worker_lps, hp, wdt, seed=21)
+    ls.run(events, check_every=0)
+    assert ls.bit_identical
+
+    dg = DeviceGenerator(lay, 21)
+    h2 = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, **hp)
+    scratch = torch.empty(lay.P, dtype=torch.float32 if wdt == gen.F32 else torch.int16, device="cuda")
+
+    def producer(index, worker, rnd):
+        return dg.worker_result(h2.peek(hb.BUF_THETA0, worker), worker, rnd, out=scratch, worker_dtype=wdt)
+
+    log = h2.replay(events, producer)
+    for name, idx in ls.all_buffers():
+        a = ls.gpu_values(name, idx)
+        which = {"Theta": hb.BUF_THETA_G, "Mg": hb.BUF_M_G, "th": hb.BUF_THETA_L, "ml": hb.BUF_M_L,
+                 "anchor": hb.BUF_ANCHOR, "outbox": hb.BUF_OUTBOX, "inbox": hb.BUF_INBOX, "th0": hb.BUF_THETA0}[name]
+        b = h2.read(which, idx)
+        assert np.array_equal(a.view(np.uint8), b.view(np.uint8)), (name, idx)
+    assert len(log) == len(ls.log)
+    for rec, want in zip(log, ls.log):
+        assert (int(rec["kind"]), int(rec["lps"]), int(rec["t"]), int(rec["t_last"]), int(rec["gps_iter"])) == \
+               (want["kind"], want["lps"], want["t"], want["t_last"], want["gps_iter"])
+        if want["kind"] == tr.ARRIVE:
+            assert int(rec["worker"]) == want["worker"]
+            assert int(rec["worker_staleness"]) == want["worker_staleness"]
+            assert bool(rec["pushed"]) == want["pushed"]
+        if want["kind"] == tr.PULL:
+            assert int(rec["gps_lag"]) == want["gps_lag"]
+    assert int(log["pushed"].sum()) == int((events["kind"] == tr.GPS_RECV).sum())
+    h2.close()
+    ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# call-order errors leave the state untouched
+# ---------------------------------------------------------------------------------------------
+def test_state_machine_errors():
+    P = 1000
+    init = torch.linspace(-1, 1, P, device="cuda")
+    h = hb.Halos(init, [0, 1], K=1, **PAPER_HP)
+    snap = lambda: [h.read(b, i).copy() for b in (hb.BUF_THETA_L, hb.BUF_M_L, hb.BUF_ANCHOR) for i in (0, 1)] + \
+                   [h.read(hb.BUF_THETA_G), h.read(hb.BUF_M_G)]
+    before, c_before = snap(), h.counters(0)
+    thH = init + 0.01
+
+    def expect(status, fn, *a):
+        with pytest.raises(hb.HalosError) as e:
+            fn(*a)
+        assert e.value.status == status
+
+    expect(hb.ERR_BAD_STATE, h.lps_apply, 0, 0)          # no pending result
+    expect(hb.ERR_BAD_STATE, h.gps_merge, 0)             # nothing pushed
+    expect(hb.ERR_BAD_STATE, h.lps_pull, 0)              # nothing answered
+    expect(hb.ERR_INVALID_ARG, h.lps_apply, 7, 0)
+    expect(hb.ERR_INVALID_ARG, h.worker_delta, 9, thH)
+    h.worker_delta(0, thH)
+    expect(hb.ERR_BAD_STATE, h.worker_delta, 0, thH)     # already pending
+    expect(hb.ERR_INVALID_ARG, h.lps_apply, 1, 0)        # worker 0 belongs to LPS 0
+    for a, b in zip(before, snap()):
+        np.testing.assert_array_equal(a, b)
+    assert h.counters(0) == c_before
+    assert h.lps_apply(0, 0) is True                     # K = 1: push due
+    h.lps_push(0)
+    expect(hb.ERR_BAD_STATE, h.lps_push, 0)              # second push while in flight
+    expect(hb.ERR_BAD_STATE, h.lps_pull, 0)
+    h.gps_merge(0)
+    expect(hb.ERR_BAD_STATE, h.gps_merge, 0)
+    h.lps_pull(0)
+    c = h.counters(0)
+    assert (c["t"], c["t_last"], c["phase"], c["i"]) == (1, 1, hb.IDLE, 1)
+    expect(hb.ERR_INVALID_ARG, h.read, hb.BUF_THETA_L, 0, P - 1, 5)
+    h.close()
+    with pytest.raises(ValueError):
+        hb.Halos(init, [0], tensor_numel=[3, 4])
+
+
+# ---------------------------------------------------------------------------------------------
+# host-resident worker results (staged copy) give the same bits as device-resident ones
+# ---------------------------------------------------------------------------------------------
+def test_host_inputs_match_device_inputs():
+    lay = layouts.flat_layout("x", 300_001)
+    init = torch.from_numpy(gen.theta_init(lay, 4)).cuda()
+    a = hb.Halos(init, [0, 0, 0], **PAPER_HP)
+    b = hb.Halos(init, [0, 0, 0], **PAPER_HP)
+    pinned = [torch.empty(lay.P, dtype=torch.float32).pin_memory() for _ in range(3)]
+    for rnd in range(3):
+        # two staging buffers: at most two host results may wait for their apply
+        for group in ((2, 0), (1,)):
+            for w in group:
+                res = gen.worker_result(a.read(hb.BUF_THETA0, w), lay, 4, w, rnd)
+                pinned[w].copy_(torch.from_numpy(res))
+                b.worker_delta_host(w, pinned[w])
+                a.worker_delta(w, torch.from_numpy(res).cuda())
+            for w in group:
+                a.lps_apply(0, w)
+                b.lps_apply(0, w)
+        np.testing.assert_array_equal(a.read(hb.BUF_THETA_L, 0), b.read(hb.BUF_THETA_L, 0))
+        np.testing.assert_array_equal(a.read(hb.BUF_THETA0, 1), b.read(hb.BUF_THETA0, 1))
+    for w in (0, 1):
+        b.worker_delta_host(w, pinned[w])
+    with pytest.raises(hb.HalosError) as e:
+        b.worker_delta_host(2, pinned[2])          # both staging buffers are taken
+    assert e.value.status == hb.ERR_BAD_STATE
+    a.close()
+    b.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# optional per-tensor squared norms
+# ---------------------------------------------------------------------------------------------
+def test_norm_statistics():
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 100000])
+    worker_lps = [0, 1]
+    ls = Lockstep(lay, worker_lps, dict(K=2, **PAPER_HP), gen.F32, seed=3, flags=hb.FLAG_STATS, chunk_elems=2048)
+    events = tr.random_trace(worker_lps, 12, 2, seed=1)
+    off = lay.offsets.astype(np.int64)
+    for ev in events:
+        rec = ls.step(ev)
+        if rec["kind"] == tr.ARRIVE:
+            np.testing.assert_allclose(ls.h.stats(0, rec["lps"]), ls.o.sq_norms("delta", rec["lps"], off), rtol=2e-6)
+            if rec["pushed"]:
+                np.testing.assert_allclose(ls.h.stats(1, rec["lps"]), ls.o.sq_norms("outbox", rec["lps"], off), rtol=2e-6)
+    ls.compare(ls.all_buffers(), FULL_TRACE_TOL)
+    assert ls.bit_identical
+    ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# LLM-shaped configurations at full size on the GPU; the oracle replays probe windows
+# ---------------------------------------------------------------------------------------------
+def _run_config(name, n_arrivals, check_every, full_every):
+    wl = workloads.workload(name)
+    probes = default_probes(wl.layout, width=4096, n_random=8, seed=wl.seed)
+    ls = Lockstep(wl.layout, wl.worker_lps, wl.hyper(), wl.worker_dtype, wl.seed, probes=probes)
+    events = wl.trace(n_arrivals)
+    ls.run(events, check_every=check_every, full_check_every=full_every)
+    assert ls.max_err <= FULL_TRACE_TOL
+    assert ls.bit_identical
+    kinds = [r["kind"] for r in ls.log]
+    assert kinds.count(tr.PULL) >= 2
+    ls.close()
+    return ls
+
+
+def test_config_70m_bf16_full_trace():
+    _run_config("70m", None, check_every=1, full_every=250)
+
+
+def test_config_160m_fp32_full_trace():
+    _run_config("160m", None, check_every=1, full_every=500)
+
+
+def test_config_410m_fp32_staleness_order():
+    # 32 workers with fp32 copies: ~89 GB on the device
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100 * (1 << 30):
+        pytest.skip("needs ~95 GB of free device memory")
+    ls = _run_config("410m", None, check_every=4, full_every=0)
+    # the slowed-down region sees the stalest workers' results least often but every LPS made round trips
+    by_lps = {}
+    for r in ls.log:
+        if r["kind"] == tr.PULL:
+            by_lps[r["lps"]] = by_lps.get(r["lps"], 0) + 1
+    assert set(by_lps) == {0, 1, 2, 3}
