@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the HALoS server-side update path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 160m] [--impl ours|reference]
+
+A step replays the next ``--events-per-step`` events (worker arrivals with their pushes, GPS
+updates, merges) of the workload's seeded asynchronous trace through the library's event-queue
+driver: one fused kernel per event over all tensors of the model.  Metric: parameters updated per
+second (every event updates the P parameters of one model).
+
+    value       device-resident: each worker's result theta_H already sits in HBM
+    e2e         the same replay through the C ABI with HOST-resident worker results (pinned), the
+                host->device copy of every result and a device->host read of a probe of the
+                models inside the timed region
+    roofline    arrive kernel (delta + LPS momentum + schedule copy): algorithmic bytes / mean
+                launch duration (CUDA events recorded by the library on its stream inside the timed
+                region) against the measured HBM copy bandwidth of this machine
+    cpu_baseline  the CPU oracle as it stands (one core) on a bounded index slice of the workload
+
+``--impl reference`` times the CPU oracle on a bounded sample and prints the same line shape.
+With N > 1 (torchrun) every rank replays the trace on its own index shard of an N-times larger
+model on its own GPU: no data-path collective; NCCL only carries the barrier and the max of the
+per-rank times.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "params_updated_per_sec"
+UNIT = "params/s"
+BYTES_PER_PARAM = {"arrive_f32": 28, "arrive_bf16": 22, "arrive_push_f32": 36, "arrive_push_bf16": 30,
+                   "push": 12, "gps": 24, "pull": 16}
+
+
+# ------------------------------------------------------------------------------------ helpers
+def measured_peak_gbs():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.2):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = None
+            try:
+                import torch
+                uuid = str(torch.cuda.get_device_properties(index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self.dev = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _names(self, mask: int):
+        nv = self.nv
+        table = [("gpu_idle", "nvmlClocksThrottleReasonGpuIdle"),
+                 ("applications_clocks_setting", "nvmlClocksThrottleReasonApplicationsClocksSetting"),
+                 ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap"),
+                 ("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("sync_boost", "nvmlClocksThrottleReasonSyncBoost"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("hw_power_brake_slowdown", "nvmlClocksThrottleReasonHwPowerBrakeSlowdown"),
+                 ("display_clock_setting", "nvmlClocksThrottleReasonDisplayClockSetting")]
+        return {n for n, attr in table if mask & int(getattr(nv, attr, 0))}
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+                self.reasons |= self._names(int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons - {"gpu_idle"})}
+
+
+def reduce_over_ranks(dist, elapsed_ms: float, units: float, device=None):
+    """(max elapsed over ranks, sum of units over ranks); identity without a process group."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return elapsed_ms, units
+    import torch
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def window_events(n_steps: int, events_per_step: int, wl):
+    """A trace long enough for n_steps windows of events_per_step events."""
+    need = n_steps * events_per_step
+    n_arr = max(wl.n_arrivals, need)
+    ev = wl.trace(n_arr)
+    while len(ev) < need:
+        n_arr = int(n_arr * 1.2) + 16
+        ev = wl.trace(n_arr)
+    return ev[:need]
+
+
+# ------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample(wl, events, slice_params: int, budget_s: float):
+    """Times the CPU oracle (as it stands, one core) replaying `events` on the index slice
+    [0, slice_params) of the workload until the time budget is used.  Returns (params/s, description)."""
+    import oracle
+    from oracle import HalosOracle
+    from paper_2506_04531_b200.inputs import gen, trace as tr
+    lay = wl.layout
+    S = min(slice_params, lay.P)
+    init = gen.theta_init(lay, wl.seed, 0, S)
+    o = HalosOracle(init, wl.worker_lps, worker_dtype=wl.worker_dtype, dtype=np.float32, **wl.hyper())
+    spent, done = 0.0, 0
+    for ev in events:
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        if kind == tr.ARRIVE:
+            r = o.worker_info(w)["round"]
+            thH = gen.worker_result(o.buffer("th0", w), lay, wl.seed, w, r, 0, S, wl.worker_dtype)   # untimed input
+            t0 = time.perf_counter()
+            o.arrive(w, thH)
+        elif kind == tr.GPS_RECV:
+            t0 = time.perf_counter()
+            o.gps_recv(l)
+        else:
+            t0 = time.perf_counter()
+            o.pull(l)
+        spent += time.perf_counter() - t0
+        done += 1
+        if spent >= budget_s:
+            break
+    o.close()
+    return done * S / spent, f"first {done} events of the trace on the index slice [0,{S}) of {lay.P} parameters", spent, done
+
+
+# ------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "410m"])
+    ap.add_argument("--events-per-step", type=int, default=128)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    ap.add_argument("--chunk-elems", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_2506_04531_b200.inputs import workloads
+    wl = workloads.workload(args.workload)
+    lay = wl.layout
+    P = lay.P
+    wname = {0: "f32", 1: "bf16"}[wl.worker_dtype]
+    config = {"workload": f"{wl.name}: decoder layout P={P} ({lay.n_tensors} tensors), {wl.n_workers} workers over "
+                          f"{wl.n_lps} LPS, 1 GPS, fp32 master + {wname} worker copies, K={wl.K}, paper hyperparameters",
+              "events_per_step": args.events_per_step, "trace_seed": wl.seed,
+              "l2": "every buffer (%.0f MB) is larger than L2; no flush needed" % (P * 4 / 1e6),
+              "parallelism": "index-sharded replicas, no collective" if world > 1 else "single GPU"}
+
+    # ---------------------------------------------------------------- reference arm = the oracle
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        events = window_events(args.steps + args.warmup, args.events_per_step, wl)
+        S = 1 << 22
+        per_step_budget = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+        rates, t_total, total_done = [], 0.0, 0
+        for s in range(args.steps + args.warmup):
+            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
+            rate, desc, spent, done = oracle_sample(wl, win, S, per_step_budget)
+            if s >= args.warmup:
+                rates.append(rate)
+                t_total += spent
+                total_done += done
+        value = total_done * S / t_total
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / max(1, args.steps),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                 "sample": f"per step: up to {per_step_budget:.0f} s of the step's events on the index slice [0,{S})"},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    # ---------------------------------------------------------------- our arm
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the update path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2506_04531_b200 import binding as hb, build as _build
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2506_04531_b200.inputs import gen
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+
+    n_steps = args.steps + args.warmup
+    events = window_events(n_steps * (1 if args.no_e2e else 2), args.events_per_step, wl)
+    seed = wl.seed + 1000 * rank                      # each rank: its own shard of a larger model
+    dgen = DeviceGenerator(lay, seed, device=dev)
+    init = dgen.theta_init()
+    h = hb.Halos(init, wl.worker_lps, lay.numel, worker_dtype=wl.worker_dtype, chunk_elems=args.chunk_elems, **wl.hyper())
+    wdt = torch.float32 if wl.worker_dtype == gen.F32 else torch.int16
+    # device-resident worker results: one buffer per worker, theta_H = Theta_0 + sigma z_w
+    results = [dgen.worker_result(h.peek(hb.BUF_THETA0, w), w, 0, worker_dtype=wl.worker_dtype)
+               for w in range(wl.n_workers)]
+    del init
+    torch.cuda.synchronize(dev)
+
+    def producer_dev(index, worker, rnd):
+        return results[worker]
+
+    def run_step(s, e2e=False, host_results=None, probe=None):
+        win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
+        if not e2e:
+            h.replay(win, producer_dev, want_log=False)
+            return 0
+        # end to end: results live in pinned host memory and are copied in by the library; two
+        # staging buffers let the copy of the next result overlap the current update kernel
+        from paper_2506_04531_b200.inputs import trace as tr
+        pend = []
+        n = len(win)
+        nxt = 0
+
+        def feed():
+            nonlocal nxt
+            while nxt < n and len(pend) < 2:
+                ev = win[nxt]
+                if int(ev["kind"]) == tr.ARRIVE:
+                    w = int(ev["worker"])
+                    if any(int(win[p]["worker"]) == w for p in pend):
+                        break
+                    h.worker_delta_host(w, host_results[w])
+                    pend.append(nxt)
+                nxt += 1
+        for k in range(n):
+            nxt = max(nxt, k)
+            feed()
+            ev = win[k]
+            kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+            if kind == tr.ARRIVE:
+                assert pend and pend[0] == k
+                pend.pop(0)
+                if h.lps_apply(l, w):
+                    h.lps_push(l)
+                feed()
+            elif kind == tr.GPS_RECV:
+                h.gps_merge(l)
+            else:
+                h.lps_pull(l)
+        # device -> host read of the step's result: a probe of the global and local models
+        got = 0
+        for which, idx in probe:
+            got += h.read(which, idx, 0, 1024).nbytes
+        return got
+
+    # ---- warm-up, then the timed region (device-resident) ----
+    for s in range(args.warmup):
+        run_step(s)
+    torch.cuda.synchronize(dev)
+    h.timing_enable(True)
+    launches0 = h.info()["launches"]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clk:
+        e0.record()
+        for s in range(args.warmup, n_steps):
+            run_step(s)
+        e1.record()
+        torch.cuda.synchronize(dev)
+    if world > 1:
+        dist.barrier()
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = h.info()["launches"] - launches0
+    timing = h.timing_read()
+    h.timing_enable(False)
+    units = float(args.steps * args.events_per_step) * P
+    t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
+    value = units_all / (t_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel ----
+    peak, peak_kind = measured_peak_gbs()
+    n_arr, ms_arr = timing["arrive"]
+    bpp = BYTES_PER_PARAM["arrive_" + wname]
+    achieved = (bpp * P / 1e9) / (ms_arr / n_arr * 1e-3) if n_arr else None
+    traffic = None
+    prof = ROOT / "profiles" / "traffic.json"
+    if prof.exists():
+        try:
+            tj = json.loads(prof.read_text())
+            key = f"arrive_{wname}"
+            if key in tj:
+                traffic = tj[key]["dram_bytes_per_param"] * P
+        except Exception:
+            pass
+    roofline = {"bound": "hbm", "kernel": f"arrive_kernel<{wname}>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": bpp * P,
+                "per_kernel": {k: {"launches": n, "mean_ms": (ms / n if n else None),
+                                   "GBps": ((BYTES_PER_PARAM.get(k, BYTES_PER_PARAM.get(k + "_" + wname, 0)) * P / 1e9) / (ms / n * 1e-3) if n else None)}
+                               for k, (n, ms) in timing.items()}}
+
+    # ---- end to end (host-resident worker results) ----
+    e2e = None
+    if not args.no_e2e:
+        host_results = [torch.empty(P, dtype=wdt).pin_memory() for _ in range(wl.n_workers)]
+        for w in range(wl.n_workers):
+            host_results[w].copy_(results[w])
+        probe = [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]
+        from paper_2506_04531_b200.inputs import trace as tr
+        e2e_steps = max(1, min(args.steps, 3))
+        base = n_steps
+        run_step(base, e2e=True, host_results=host_results, probe=probe)            # warm-up (allocates staging)
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        d2h = 0
+        arrivals = 0
+        for s in range(base + 1, base + 1 + e2e_steps):
+            d2h = run_step(s, e2e=True, host_results=host_results, probe=probe)
+            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
+            arrivals += int((win["kind"] == tr.ARRIVE).sum())
+        torch.cuda.synchronize(dev)
+        dt_ms = (time.perf_counter() - t0) * 1e3
+        u = float(e2e_steps * args.events_per_step) * P
+        dt_ms, u_all = reduce_over_ranks(dist if world > 1 else None, dt_ms, u, dev)
+        e2e = {"value": u_all / (dt_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(arrivals / e2e_steps * P * (4 if wl.worker_dtype == gen.F32 else 2)),
+               "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps}
+        del host_results
+
+    h.close()
+    del results
+    torch.cuda.empty_cache()
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rate, desc, spent, done = oracle_sample(wl, events, 1 << 22, args.cpu_budget_s)
+        cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc + f" ({spent:.1f} s)"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": t_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
