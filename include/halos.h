@@ -215,6 +215,30 @@ enum {
 int halos_timing_enable(halos_ctx* ctx, int on);
 int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double* total_ms);
 
+/* Push step for callers that must not allocate.  (The paper has no counterpart: this is a
+ * deployment variant of Alg. 1 line 14 as computed by halos_lps_push with HALOS_FLAG_STATS.)
+ *
+ *   Delta_dev[j] = theta_dev[j] - anchor_dev[j]  for j < n,   *sqnorm_dev = sum_j Delta_dev[j]^2
+ *
+ * Meant for code that runs where device allocation is off limits: while a memory pool is frozen
+ * or full, in sections where an allocator call could block or synchronise the device, or under a
+ * policy of no cudaMalloc after start-up.  It needs no context; inputs and outputs are the caller's
+ * (device pointers on `device`, fp32 arrays of n elements, 4-byte aligned -- 16-byte alignment of all
+ * three enables the vector path; sqnorm_dev points to one double).  The reduction scratch is a fixed
+ * 512 KB array inside the library, present on every GPU that loads it until the process exits, which
+ * caps n at HALOS_NOALLOC_MAX_ELEMS: larger n returns HALOS_ERR_UNSUPPORTED and touches nothing.
+ * The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine) and enqueues
+ * two kernels on `stream` (cudaStream_t, NULL = legacy default stream); it does not wait for them.
+ * The first call on each device looks up the scratch array's device address (cudaGetSymbolAddress)
+ * and should therefore be made before any stream capture begins.  All calls share the scratch,
+ * which keeps the previous call's partial sums; each call overwrites every slot it later reads, so
+ * nothing needs clearing, but calls that overlap on the GPU race on it: keep them on one stream or
+ * otherwise serialised.  Returns HALOS_OK, HALOS_ERR_UNSUPPORTED (n too large),
+ * HALOS_ERR_INVALID_ARG (null/misaligned pointer, bad device) or HALOS_ERR_CUDA. */
+#define HALOS_NOALLOC_MAX_ELEMS (1ull << 29)
+int halos_push_noalloc(int32_t device, void* stream, const float* theta_dev, const float* anchor_dev,
+                       float* Delta_dev, uint64_t n, double* sqnorm_dev);
+
 const char* halos_strerror(int status);
 /* Text of the last error on this context (or of the last failed halos_create when ctx is NULL). */
 const char* halos_last_error(halos_ctx* ctx);

@@ -28,8 +28,9 @@ EXPORTED = (
     "halos_default_config", "halos_create", "halos_worker_delta", "halos_worker_delta_host", "halos_lps_apply",
     "halos_lps_push", "halos_gps_merge", "halos_lps_pull", "halos_destroy", "halos_replay", "halos_peek",
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
-    "halos_timing_read", "halos_strerror", "halos_last_error",
+    "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc",
 )
+NOALLOC_MAX_ELEMS = 1 << 29
 
 ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
 FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
@@ -99,6 +100,7 @@ def load_library():
     lib.halos_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u32), C.POINTER(u32), C.POINTER(u64)]
     lib.halos_timing_enable.argtypes = [vp, i32]
     lib.halos_timing_read.argtypes = [vp, u32, C.POINTER(u64), C.POINTER(C.c_double)]
+    lib.halos_push_noalloc.argtypes = [C.c_int32, vp, vp, vp, vp, u64, vp]
     lib.halos_strerror.argtypes = [i32]
     lib.halos_strerror.restype = C.c_char_p
     lib.halos_last_error.argtypes = [vp]
@@ -121,6 +123,22 @@ def _ptr(x) -> Optional[int]:
     if isinstance(x, np.ndarray):
         return x.ctypes.data
     raise TypeError(type(x))
+
+
+def push_noalloc(theta, anchor, Delta_out, sqnorm_out, n=None, stream=None) -> int:
+    """Delta_out = theta - anchor and sqnorm_out[0] = sum Delta^2 without any allocation by the library.
+
+    For callers that cannot allocate device memory (frozen or full pools, no-cudaMalloc policies):
+    all four tensors are the caller's (fp32 CUDA tensors / raw addresses, sqnorm_out one float64).
+    Returns the status code instead of raising so that the size limit (NOALLOC_MAX_ELEMS ->
+    ERR_UNSUPPORTED) can be handled by the caller.  Calls share one fixed scratch array inside the
+    library: do not let two of them overlap on the GPU."""
+    import torch
+    lib = load_library()
+    n = int(theta.numel()) if n is None else int(n)
+    dev = theta.device.index if hasattr(theta, "device") and theta.device.index is not None else torch.cuda.current_device()
+    st = (stream if stream is not None else torch.cuda.current_stream(dev)).cuda_stream
+    return int(lib.halos_push_noalloc(dev, st, _ptr(theta), _ptr(anchor), _ptr(Delta_out), n, _ptr(sqnorm_out)))
 
 
 class Halos:

@@ -20,7 +20,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
 TARGETS = {
-    "halos": dict(out=PKG / "libhalos_b200.so", src=[PKG / "csrc" / "halos.cu"],
+    "halos": dict(out=PKG / "libhalos_b200.so", src=[PKG / "csrc" / "halos.cu", PKG / "csrc" / "halos_noalloc.cu"],
                   deps=[PKG / "csrc" / "halos_kernels.cuh", INCLUDE / "halos.h"]),
     "inputs": dict(out=PKG / "inputs" / "libhalos_inputs.so", src=[PKG / "inputs" / "csrc" / "synth_inputs.cu"],
                    deps=[]),
