@@ -184,7 +184,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "410m"])
+    ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "410m", "70m_f32_small"])
     ap.add_argument("--events-per-step", type=int, default=128)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -58,7 +58,7 @@ class Workload:
 
 
 def workload(name: str) -> Workload:
-    """toy | toy_k4 | 70m | 160m | 410m  (hyperparameters: the paper's selected values)."""
+    """toy | toy_k4 | 70m | 160m | 410m | 70m_f32_small  (hyperparameters: the paper's selected values)."""
     if name == "toy":
         return Workload("toy", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1)
     if name == "toy_k4":
@@ -70,6 +70,10 @@ def workload(name: str) -> Workload:
     if name == "410m":
         return Workload("410m", named_layout("410m"), 32, 4, gen.F32, 1589.7, 2000, seed=4,
                         slow_region_factor=3.0)
+    if name == "70m_f32_small":
+        # profiling case: 70M layout, fp32 copies, 2 workers on 1 LPS (~3 GB on the device, every
+        # buffer still larger than L2); K=8 so that pushes, GPS updates and merges occur early
+        return Workload("70m_f32_small", named_layout("70m"), 2, 1, gen.F32, 238.4, 200, seed=6, K=8)
     raise KeyError(name)
 
 
