@@ -12,8 +12,11 @@ from typing import Callable, Optional, Sequence
 
 import numpy as np
 
+import os
+
 _PKG = Path(__file__).resolve().parent
-LIB_PATH = _PKG / "libhalos_b200.so"
+# HALOS_B200_LIB points at an alternative build of the same library (kernel tuning experiments).
+LIB_PATH = Path(os.environ.get("HALOS_B200_LIB", _PKG / "libhalos_b200.so"))
 
 OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED = range(6)
 F32, BF16 = 0, 1

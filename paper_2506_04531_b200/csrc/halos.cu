@@ -15,8 +15,8 @@ using namespace halos;
 namespace {
 
 constexpr uint32_t kDefaultChunkElems = 8192;
-constexpr int kUnroll = 4;
-constexpr bool kStream = true;
+constexpr int kUnroll = HALOS_UNROLL;
+constexpr bool kStream = HALOS_STREAM_HINT != 0;
 constexpr int kStageSlots = 2;
 
 thread_local std::string g_create_error;

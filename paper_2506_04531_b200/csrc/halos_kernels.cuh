@@ -29,7 +29,17 @@ struct Chunk {
     uint32_t tensor;           // tensor the chunk belongs to
 };
 
-constexpr int kThreads = 256;
+// Compile-time tuning knobs (the defaults are the measured best on B200; see profiles/).
+#ifndef HALOS_THREADS
+#define HALOS_THREADS 256
+#endif
+#ifndef HALOS_UNROLL
+#define HALOS_UNROLL 4
+#endif
+#ifndef HALOS_STREAM_HINT
+#define HALOS_STREAM_HINT 1
+#endif
+constexpr int kThreads = HALOS_THREADS;
 
 // ---------------------------------------------------------------- element helpers
 __device__ __forceinline__ void model_update(float& x, float& m, float d, float eta, float beta, float omb) {
