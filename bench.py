@@ -43,6 +43,10 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {"arrive_f32": 28, "arrive_bf16": 22, "arrive_push_f32": 36, "arrive_push_bf16": 30,
                    "push": 12, "gps": 24, "pull": 16}
 
+# DRAM read+write bytes per parameter per launch from the ncu capture summarised in
+# profiles/ncu_full_kernels_70m_f32_small.md (P = 70,426,624; traffic is proportional to P).
+DRAM_BYTES_PER_PARAM = {"arrive_f32": 27.22, "arrive_push_f32": 35.23, "gps": 23.20, "pull": 15.20}
+
 
 # ------------------------------------------------------------------------------------ helpers
 def measured_peak_gbs():
@@ -177,6 +181,80 @@ def oracle_sample(wl, events, slice_params: int, budget_s: float):
     return done * S / spent, f"first {done} events of the trace on the index slice [0,{S}) of {lay.P} parameters", spent, done
 
 
+# ------------------------------------------------------------------------------------ bandwidth sweep
+def run_sweep(args):
+    """Configuration 5: flat fp32 buffers from 2^20 to 2^30 parameters plus the 1.4B-class decoder layout;
+    per size one context with 1 LPS / 1 worker, cycles of {arrive, arrive+due, push, gps, pull}, each kernel
+    timed by the library's CUDA events.  Sizes whose working set is below 512 MB rotate over several
+    contexts so that consecutive launches do not find their data in L2."""
+    import torch
+    from paper_2506_04531_b200 import binding as hb, build as _build
+    from paper_2506_04531_b200.inputs import gen, layouts, workloads
+    _build.build()
+    dev = torch.device("cuda", 0)
+    peak, peak_kind = measured_peak_gbs()
+    cases = [(f"flat_{n}", layouts.flat_layout("flat", n)) for n in workloads.SWEEP_SIZES]
+    cases.append(("decoder_1p4b", layouts.named_layout("1p4b")))
+    rows = []
+    for wdt, wname in ((gen.F32, "f32"), (gen.BF16, "bf16")):
+        for name, lay in cases:
+            P = lay.P
+            if args.sweep_max and P > args.sweep_max:
+                continue
+            wb = 4 if wdt == gen.F32 else 2
+            set_bytes = P * (6 * 4 + 3 * wb)
+            n_sets = max(1, min(64, -(-(512 << 20) // set_bytes)))
+            ctxs, ths = [], []
+            for k in range(n_sets):
+                init = torch.randn(P, device=dev) * 0.02
+                ctxs.append(hb.Halos(init, [0], lay.numel, K=2, worker_dtype=wdt, chunk_elems=args.chunk_elems))
+                th = init + 1e-3 * torch.randn(P, device=dev)
+                ths.append(th if wdt == gen.F32 else th.to(torch.bfloat16).view(torch.int16))
+                del init, th
+
+            def a1(h, th):
+                h.worker_delta(0, th); h.lps_apply(0, 0)
+
+            def a2(h, th):
+                h.worker_delta(0, th)
+                assert h.lps_apply(0, 0)
+
+            phases = (a1, a2, lambda h, th: h.lps_push(0), lambda h, th: h.gps_merge(0), lambda h, th: h.lps_pull(0))
+
+            def cycle():
+                # kind-major order: between two launches on the same context all other contexts run,
+                # so small sizes do not find their buffers in L2
+                for ph in phases:
+                    for h, th in zip(ctxs, ths):
+                        ph(h, th)
+
+            reps = max(3, min(40, int(2e9 // max(1, P * n_sets))))
+            cycle()
+            torch.cuda.synchronize(dev)
+            for h in ctxs:
+                h.timing_enable(True)
+            for _ in range(reps):
+                cycle()
+            agg = {}
+            for h in ctxs:
+                for k, (n, ms) in h.timing_read().items():
+                    a = agg.setdefault(k, [0, 0.0]); a[0] += n; a[1] += ms
+                h.close()
+            B = {"arrive": 16 + 3 * wb, "push": 12, "gps": 24, "pull": 16}
+            row = {"case": name, "P": P, "tensors": lay.n_tensors, "worker_dtype": wname, "buffer_MB": P * 4 / 1e6,
+                   "contexts_rotated": n_sets}
+            for k in ("arrive", "push", "gps", "pull"):
+                n, ms = agg[k]
+                t = ms / n * 1e-3
+                row[k] = {"us": t * 1e6, "GBps": B[k] * P / 1e9 / t, "frac_of_measured": B[k] * P / 1e9 / t / peak,
+                          "Gparams_per_s": P / t / 1e9}
+            rows.append(row)
+            del ctxs, ths
+            torch.cuda.empty_cache()
+    print(json.dumps({"sweep": rows, "peak_GBps": peak, "peak_source": peak_kind, "metric": METRIC}))
+    return 0
+
+
 # ------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -190,7 +268,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--chunk-elems", type=int, default=0)
+    ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over buffer sizes instead of the default line")
+    ap.add_argument("--sweep-max", type=int, default=0, help="largest size to include (0 = all)")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
@@ -345,16 +427,8 @@ def main():
     n_arr, ms_arr = timing["arrive"]
     bpp = BYTES_PER_PARAM["arrive_" + wname]
     achieved = (bpp * P / 1e9) / (ms_arr / n_arr * 1e-3) if n_arr else None
-    traffic = None
-    prof = ROOT / "profiles" / "traffic.json"
-    if prof.exists():
-        try:
-            tj = json.loads(prof.read_text())
-            key = f"arrive_{wname}"
-            if key in tj:
-                traffic = tj[key]["dram_bytes_per_param"] * P
-        except Exception:
-            pass
+    tpp = DRAM_BYTES_PER_PARAM.get("arrive_" + wname)
+    traffic = tpp * P if tpp else None
     roofline = {"bound": "hbm", "kernel": f"arrive_kernel<{wname}>", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": bpp * P,

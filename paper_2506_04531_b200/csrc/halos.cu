@@ -14,9 +14,10 @@ using namespace halos;
 
 namespace {
 
-constexpr uint32_t kDefaultChunkElems = 8192;
+constexpr uint32_t kDefaultChunkElems = kThreads * kVecElems * HALOS_UNROLL;  // one batch of loads per CTA: 4096
 constexpr int kUnroll = HALOS_UNROLL;
 constexpr bool kStream = HALOS_STREAM_HINT != 0;
+constexpr int kVE = kVecElems;
 constexpr int kStageSlots = 2;
 
 thread_local std::string g_create_error;
@@ -147,15 +148,15 @@ void release(halos_ctx* c) {
     (void)cudaGetLastError();
 }
 
-// The chunk table: each tensor is cut into an unaligned head (0-3 elements, so that everything
-// after it starts on a 16-byte boundary of the packed fp32 state), full chunks, and a tail.
+// The chunk table: each tensor is cut into an unaligned head (fewer than kVecElems elements, so that
+// everything after it starts on a vector boundary of the packed state), full chunks, and a tail.
 void build_chunks(halos_ctx* c, uint32_t chunk_elems) {
     c->chunks.clear();
     c->tensor_chunk_begin.assign(c->tensor_numel.size() + 1, 0);
     for (size_t k = 0; k < c->tensor_numel.size(); ++k) {
         c->tensor_chunk_begin[k] = (uint32_t)c->chunks.size();
         uint64_t pos = c->tensor_off[k], end = c->tensor_off[k] + c->tensor_numel[k];
-        uint64_t head = (4 - (pos & 3)) & 3;
+        uint64_t head = (kVE - (pos % kVE)) % kVE;
         if (head && pos < end) {
             uint64_t n = head < end - pos ? head : end - pos;
             c->chunks.push_back(Chunk{pos, (uint32_t)n, (uint32_t)k});
@@ -215,11 +216,11 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
     if (push) {
-        if (stats) arrive_kernel<W, true, true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_kernel<W, true, false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (stats) arrive_kernel<W, true, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_kernel<W, true, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     } else {
-        if (stats) arrive_kernel<W, false, true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_kernel<W, false, false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (stats) arrive_kernel<W, false, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_kernel<W, false, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     }
     tm.stop();
     c->launches++;
@@ -310,7 +311,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     for (uint32_t w = 0; w < cfg->n_workers; ++w)
         if (cfg->worker_lps[w] >= cfg->n_lps) return fail(nullptr, HALOS_ERR_INVALID_ARG, "worker_lps[%u] out of range", w);
     uint32_t chunk_elems = cfg->chunk_elems ? cfg->chunk_elems : kDefaultChunkElems;
-    if (chunk_elems % 4 != 0 || chunk_elems < 4) return fail(nullptr, HALOS_ERR_INVALID_ARG, "chunk_elems must be a positive multiple of 4");
+    if (chunk_elems % 8 != 0) return fail(nullptr, HALOS_ERR_INVALID_ARG, "chunk_elems must be a positive multiple of 8");
 
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
@@ -504,8 +505,8 @@ int halos_lps_push(halos_ctx* c, uint32_t lps) {
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
     Timer tm(c, HALOS_K_PUSH);
-    if (stats) push_kernel<true, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-    else push_kernel<false, kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (stats) push_kernel<true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    else push_kernel<false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
@@ -527,7 +528,7 @@ int halos_gps_merge(halos_ctx* c, uint32_t lps) {
     GpsArgs a{s.outbox, c->Theta, c->Mg, s.inbox, c->cfg.eta_g, c->cfg.beta_g, 1.0f - c->cfg.beta_g};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     Timer tm(c, HALOS_K_GPS);
-    gps_kernel<kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    gps_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
@@ -546,7 +547,7 @@ int halos_lps_pull(halos_ctx* c, uint32_t lps) {
     PullArgs a{s.th, s.inbox, s.anchor, c->cfg.alpha, 1.0f - c->cfg.alpha};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     Timer tm(c, HALOS_K_PULL);
-    pull_kernel<kUnroll, kStream><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    pull_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());

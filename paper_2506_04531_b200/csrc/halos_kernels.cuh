@@ -3,7 +3,7 @@
 // One launch walks every tensor of the model through a chunk table built at context creation
 // (the multi-tensor chunk scheduler): chunk c = {begin, count, tensor} is a run of `count`
 // consecutive elements of the packed state starting at global element `begin`, never crossing a
-// tensor boundary.  One CTA processes one chunk.  Inside a chunk every thread moves 128-bit
+// tensor boundary.  One CTA processes one chunk.  Inside a chunk every thread moves 128- or 256-bit
 // vectors; all loads of an unrolled batch are issued before the first use so that each SM keeps
 // several tens of KB in flight.  Every buffer is read once and written once per event; the
 // displacement delta, the momentum update, the model update, the worker's new start snapshot and
@@ -29,17 +29,24 @@ struct Chunk {
     uint32_t tensor;           // tensor the chunk belongs to
 };
 
-// Compile-time tuning knobs (the defaults are the measured best on B200; see profiles/).
+// Compile-time tuning knobs.  The defaults are the best of a sweep on B200 over threads {128, 256, 512},
+// unroll {1, 2, 4, 8}, vector width {128, 256 bit}, evict-first hints {on, off} and chunk sizes
+// 2048..65536 on a 162M-parameter buffer: 512 threads x one 256-bit vector per stream per thread
+// (a CTA covers exactly one 4096-element chunk in a single batch of loads), no cache hints.
 #ifndef HALOS_THREADS
-#define HALOS_THREADS 256
+#define HALOS_THREADS 512
 #endif
 #ifndef HALOS_UNROLL
-#define HALOS_UNROLL 4
+#define HALOS_UNROLL 1
 #endif
 #ifndef HALOS_STREAM_HINT
-#define HALOS_STREAM_HINT 1
+#define HALOS_STREAM_HINT 0
+#endif
+#ifndef HALOS_VEC_ELEMS
+#define HALOS_VEC_ELEMS 8
 #endif
 constexpr int kThreads = HALOS_THREADS;
+constexpr int kVecElems = HALOS_VEC_ELEMS;   // elements per thread per access; chunks start on this boundary
 
 // ---------------------------------------------------------------- element helpers
 __device__ __forceinline__ void model_update(float& x, float& m, float d, float eta, float beta, float omb) {
@@ -56,49 +63,133 @@ __device__ __forceinline__ uint32_t bf16_narrow(float x) {
     return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x));  // round to nearest even
 }
 
-// ---------------------------------------------------------------- 128-bit streaming access
-// State is touched once per event and the working set is far larger than L2: evict-first hints.
-template <bool STREAM>
-__device__ __forceinline__ float4 ld4(const float* p) {
-    return STREAM ? __ldcs(reinterpret_cast<const float4*>(p)) : *reinterpret_cast<const float4*>(p);
+// ---------------------------------------------------------------- vector streaming access
+// A thread moves VE consecutive elements per access: VE = 4 -> 128-bit (float4 / 4 x bf16 in 64 bits),
+// VE = 8 -> 256-bit (ld/st.global.v8.f32, new with sm_100; 8 x bf16 in 128 bits).  Wider accesses
+// halve the number of memory requests per byte.  State is touched once per event and the working
+// set is far larger than L2, hence the evict-first (.cs) variants when STREAM is set.
+template <int VE> struct FVec { float v[VE]; };
+
+template <int VE, bool STREAM> __device__ __forceinline__ FVec<VE> ldf(const float* p);
+template <int VE, bool STREAM> __device__ __forceinline__ void stf(float* p, const FVec<VE>& r);
+
+template <> __device__ __forceinline__ FVec<4> ldf<4, true>(const float* p) {
+    float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    return FVec<4>{{t.x, t.y, t.z, t.w}};
 }
-template <bool STREAM>
-__device__ __forceinline__ void st4(float* p, float4 v) {
-    if (STREAM) __stcs(reinterpret_cast<float4*>(p), v);
-    else *reinterpret_cast<float4*>(p) = v;
+template <> __device__ __forceinline__ FVec<4> ldf<4, false>(const float* p) {
+    float4 t = *reinterpret_cast<const float4*>(p);
+    return FVec<4>{{t.x, t.y, t.z, t.w}};
 }
-template <bool STREAM>
-__device__ __forceinline__ uint2 ld4h(const uint16_t* p) {  // four bf16
-    return STREAM ? __ldcs(reinterpret_cast<const uint2*>(p)) : *reinterpret_cast<const uint2*>(p);
+template <> __device__ __forceinline__ void stf<4, true>(float* p, const FVec<4>& r) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(r.v[0], r.v[1], r.v[2], r.v[3]));
 }
-template <bool STREAM>
-__device__ __forceinline__ void st4h(uint16_t* p, uint2 v) {
-    if (STREAM) __stcs(reinterpret_cast<uint2*>(p), v);
-    else *reinterpret_cast<uint2*>(p) = v;
+template <> __device__ __forceinline__ void stf<4, false>(float* p, const FVec<4>& r) {
+    *reinterpret_cast<float4*>(p) = make_float4(r.v[0], r.v[1], r.v[2], r.v[3]);
 }
-__device__ __forceinline__ float4 widen4(uint2 v) {
-    return make_float4(bf16_widen(v.x & 0xffffu), bf16_widen(v.x >> 16), bf16_widen(v.y & 0xffffu),
-                       bf16_widen(v.y >> 16));
+template <> __device__ __forceinline__ FVec<8> ldf<8, true>(const float* p) {
+    FVec<8> r;
+    asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p));
+    return r;
 }
-__device__ __forceinline__ uint2 narrow4(float4 v) {
-    return make_uint2(bf16_narrow(v.x) | (bf16_narrow(v.y) << 16), bf16_narrow(v.z) | (bf16_narrow(v.w) << 16));
+template <> __device__ __forceinline__ FVec<8> ldf<8, false>(const float* p) {
+    FVec<8> r;
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+template <> __device__ __forceinline__ void stf<8, true>(float* p, const FVec<8>& r) {
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]),
+                 "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+                 : "memory");
+}
+template <> __device__ __forceinline__ void stf<8, false>(float* p, const FVec<8>& r) {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]),
+                 "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+                 : "memory");
+}
+
+// bf16 rows: VE 16-bit patterns = VE/2 32-bit words
+template <int VE, bool STREAM> __device__ __forceinline__ FVec<VE> ldh(const uint16_t* p);
+template <int VE, bool STREAM> __device__ __forceinline__ void sth(uint16_t* p, const FVec<VE>& r);
+template <int NW>
+__device__ __forceinline__ void widen_words(const uint32_t* w, float* out) {
+#pragma unroll
+    for (int k = 0; k < NW; ++k) {
+        out[2 * k] = bf16_widen(w[k] & 0xffffu);
+        out[2 * k + 1] = bf16_widen(w[k] >> 16);
+    }
+}
+template <int NW>
+__device__ __forceinline__ void narrow_words(const float* in, uint32_t* w) {
+#pragma unroll
+    for (int k = 0; k < NW; ++k) w[k] = bf16_narrow(in[2 * k]) | (bf16_narrow(in[2 * k + 1]) << 16);
+}
+template <> __device__ __forceinline__ FVec<4> ldh<4, true>(const uint16_t* p) {
+    uint2 t = __ldcs(reinterpret_cast<const uint2*>(p));
+    uint32_t w[2] = {t.x, t.y};
+    FVec<4> r;
+    widen_words<2>(w, r.v);
+    return r;
+}
+template <> __device__ __forceinline__ FVec<4> ldh<4, false>(const uint16_t* p) {
+    uint2 t = *reinterpret_cast<const uint2*>(p);
+    uint32_t w[2] = {t.x, t.y};
+    FVec<4> r;
+    widen_words<2>(w, r.v);
+    return r;
+}
+template <> __device__ __forceinline__ FVec<8> ldh<8, true>(const uint16_t* p) {
+    uint4 t = __ldcs(reinterpret_cast<const uint4*>(p));
+    uint32_t w[4] = {t.x, t.y, t.z, t.w};
+    FVec<8> r;
+    widen_words<4>(w, r.v);
+    return r;
+}
+template <> __device__ __forceinline__ FVec<8> ldh<8, false>(const uint16_t* p) {
+    uint4 t = *reinterpret_cast<const uint4*>(p);
+    uint32_t w[4] = {t.x, t.y, t.z, t.w};
+    FVec<8> r;
+    widen_words<4>(w, r.v);
+    return r;
+}
+template <> __device__ __forceinline__ void sth<4, true>(uint16_t* p, const FVec<4>& r) {
+    uint32_t w[2];
+    narrow_words<2>(r.v, w);
+    __stcs(reinterpret_cast<uint2*>(p), make_uint2(w[0], w[1]));
+}
+template <> __device__ __forceinline__ void sth<4, false>(uint16_t* p, const FVec<4>& r) {
+    uint32_t w[2];
+    narrow_words<2>(r.v, w);
+    *reinterpret_cast<uint2*>(p) = make_uint2(w[0], w[1]);
+}
+template <> __device__ __forceinline__ void sth<8, true>(uint16_t* p, const FVec<8>& r) {
+    uint32_t w[4];
+    narrow_words<4>(r.v, w);
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+}
+template <> __device__ __forceinline__ void sth<8, false>(uint16_t* p, const FVec<8>& r) {
+    uint32_t w[4];
+    narrow_words<4>(r.v, w);
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // worker-dtype traits: W = float (fp32 copies) or uint16_t (bf16 copies)
 template <class W> struct WTraits;
 template <> struct WTraits<float> {
-    template <bool S> static __device__ __forceinline__ float4 load4(const float* p) { return ld4<S>(p); }
-    template <bool S> static __device__ __forceinline__ void store4(float* p, float4 v) { st4<S>(p, v); }
+    template <int VE, bool S> static __device__ __forceinline__ FVec<VE> load(const float* p) { return ldf<VE, S>(p); }
+    template <int VE, bool S> static __device__ __forceinline__ void store(float* p, const FVec<VE>& v) { stf<VE, S>(p, v); }
     static __device__ __forceinline__ float load1(const float* p) { return *p; }
     static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
-    static constexpr uintptr_t kVecAlignMask = 15;
 };
 template <> struct WTraits<uint16_t> {
-    template <bool S> static __device__ __forceinline__ float4 load4(const uint16_t* p) { return widen4(ld4h<S>(p)); }
-    template <bool S> static __device__ __forceinline__ void store4(uint16_t* p, float4 v) { st4h<S>(p, narrow4(v)); }
+    template <int VE, bool S> static __device__ __forceinline__ FVec<VE> load(const uint16_t* p) { return ldh<VE, S>(p); }
+    template <int VE, bool S> static __device__ __forceinline__ void store(uint16_t* p, const FVec<VE>& v) { sth<VE, S>(p, v); }
     static __device__ __forceinline__ float load1(const uint16_t* p) { return bf16_widen(*p); }
     static __device__ __forceinline__ void store1(uint16_t* p, float v) { *p = (uint16_t)bf16_narrow(v); }
-    static constexpr uintptr_t kVecAlignMask = 7;
 };
 
 // ---------------------------------------------------------------- block reduction (statistics only)
@@ -135,8 +226,15 @@ struct ArriveArgs {
     float eta, beta, omb;
 };
 
-template <class W, bool PUSH, bool STATS, int UNROLL, bool STREAM>
-__global__ void __launch_bounds__(kThreads)
+template <int VE>
+__device__ __forceinline__ float sumsq(const FVec<VE>& d, float acc) {
+#pragma unroll
+    for (int e = 0; e < VE; ++e) acc = fmaf(d.v[e], d.v[e], acc);
+    return acc;
+}
+
+template <class W, bool PUSH, bool STATS, int UNROLL, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
     using T = WTraits<W>;
     const Chunk c = chunks[blockIdx.x];
@@ -149,55 +247,54 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
     const float eta = a.eta, beta = a.beta, omb = a.omb;
     float acc_d = 0.f, acc_D = 0.f;
 
-    const bool vec_ok = ((c.begin & 3ull) == 0) && ((reinterpret_cast<uintptr_t>(h) & T::kVecAlignMask) == 0);
+    // vector path: the chunk starts on a VE-element boundary of the packed state (bases are 256-byte
+    // aligned) and the caller's theta_H pointer is aligned to one vector of its own type
+    const bool vec_ok = ((c.begin % VE) == 0) && ((reinterpret_cast<uintptr_t>(h) % (VE * sizeof(W))) == 0);
     uint32_t done = 0;
     if (vec_ok) {
-        const uint32_t nvec = c.count >> 2;
+        const uint32_t nvec = c.count / VE;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
-            float4 vh[UNROLL], vs[UNROLL], vx[UNROLL], vm[UNROLL], va[UNROLL];
+            FVec<VE> vh[UNROLL], vs[UNROLL], vx[UNROLL], vm[UNROLL], va[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    vh[u] = T::template load4<STREAM>(h + 4ull * v);
-                    vs[u] = T::template load4<STREAM>(s0 + 4ull * v);
-                    vx[u] = ld4<STREAM>(th + 4ull * v);
-                    vm[u] = ld4<STREAM>(ml + 4ull * v);
-                    if (PUSH) va[u] = ld4<STREAM>(an + 4ull * v);
+                    const size_t o = (size_t)VE * v;
+                    vh[u] = T::template load<VE, STREAM>(h + o);
+                    vs[u] = T::template load<VE, STREAM>(s0 + o);
+                    vx[u] = ldf<VE, STREAM>(th + o);
+                    vm[u] = ldf<VE, STREAM>(ml + o);
+                    if (PUSH) va[u] = ldf<VE, STREAM>(an + o);
                 }
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    float4 d;
-                    d.x = __fsub_rn(vh[u].x, vs[u].x);
-                    d.y = __fsub_rn(vh[u].y, vs[u].y);
-                    d.z = __fsub_rn(vh[u].z, vs[u].z);
-                    d.w = __fsub_rn(vh[u].w, vs[u].w);
-                    model_update(vx[u].x, vm[u].x, d.x, eta, beta, omb);
-                    model_update(vx[u].y, vm[u].y, d.y, eta, beta, omb);
-                    model_update(vx[u].z, vm[u].z, d.z, eta, beta, omb);
-                    model_update(vx[u].w, vm[u].w, d.w, eta, beta, omb);
-                    st4<STREAM>(th + 4ull * v, vx[u]);
-                    st4<STREAM>(ml + 4ull * v, vm[u]);
-                    T::template store4<STREAM>(s0 + 4ull * v, vx[u]);
-                    if (STATS) acc_d = fmaf(d.x, d.x, fmaf(d.y, d.y, fmaf(d.z, d.z, fmaf(d.w, d.w, acc_d))));
+                    const size_t o = (size_t)VE * v;
+                    FVec<VE> d;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) {
+                        d.v[e] = __fsub_rn(vh[u].v[e], vs[u].v[e]);
+                        model_update(vx[u].v[e], vm[u].v[e], d.v[e], eta, beta, omb);
+                    }
+                    stf<VE, STREAM>(th + o, vx[u]);
+                    stf<VE, STREAM>(ml + o, vm[u]);
+                    T::template store<VE, STREAM>(s0 + o, vx[u]);
+                    if (STATS) acc_d = sumsq<VE>(d, acc_d);
                     if (PUSH) {
-                        float4 D;
-                        D.x = __fsub_rn(vx[u].x, va[u].x);
-                        D.y = __fsub_rn(vx[u].y, va[u].y);
-                        D.z = __fsub_rn(vx[u].z, va[u].z);
-                        D.w = __fsub_rn(vx[u].w, va[u].w);
-                        st4<STREAM>(ob + 4ull * v, D);
-                        if (STATS) acc_D = fmaf(D.x, D.x, fmaf(D.y, D.y, fmaf(D.z, D.z, fmaf(D.w, D.w, acc_D))));
+                        FVec<VE> D;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx[u].v[e], va[u].v[e]);
+                        stf<VE, STREAM>(ob + o, D);
+                        if (STATS) acc_D = sumsq<VE>(D, acc_D);
                     }
                 }
             }
         }
-        done = nvec << 2;
+        done = nvec * VE;
     }
-    // ragged tail (or a whole chunk whose pointers do not share 16-byte alignment): scalar
+    // ragged tail (or a whole chunk whose pointers do not share the vector alignment): scalar
     for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
         float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
         float x = th[j], m = ml[j];
@@ -234,7 +331,7 @@ struct PushArgs {
     double* partial_Delta;
 };
 
-template <bool STATS, int UNROLL, bool STREAM>
+template <bool STATS, int UNROLL, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads)
 push_kernel(const Chunk* __restrict__ chunks, PushArgs a) {
     const Chunk c = chunks[blockIdx.x];
@@ -243,33 +340,31 @@ push_kernel(const Chunk* __restrict__ chunks, PushArgs a) {
     float* ob = a.outbox + c.begin;
     float acc = 0.f;
     uint32_t done = 0;
-    if ((c.begin & 3ull) == 0) {
-        const uint32_t nvec = c.count >> 2;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
-            float4 vx[UNROLL], va[UNROLL];
+            FVec<VE> vx[UNROLL], va[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    vx[u] = ld4<STREAM>(th + 4ull * v);
-                    va[u] = ld4<STREAM>(an + 4ull * v);
+                    vx[u] = ldf<VE, STREAM>(th + (size_t)VE * v);
+                    va[u] = ldf<VE, STREAM>(an + (size_t)VE * v);
                 }
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    float4 D;
-                    D.x = __fsub_rn(vx[u].x, va[u].x);
-                    D.y = __fsub_rn(vx[u].y, va[u].y);
-                    D.z = __fsub_rn(vx[u].z, va[u].z);
-                    D.w = __fsub_rn(vx[u].w, va[u].w);
-                    st4<STREAM>(ob + 4ull * v, D);
-                    if (STATS) acc = fmaf(D.x, D.x, fmaf(D.y, D.y, fmaf(D.z, D.z, fmaf(D.w, D.w, acc))));
+                    FVec<VE> D;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx[u].v[e], va[u].v[e]);
+                    stf<VE, STREAM>(ob + (size_t)VE * v, D);
+                    if (STATS) acc = sumsq<VE>(D, acc);
                 }
             }
         }
-        done = nvec << 2;
+        done = nvec * VE;
     }
     for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
         float D = __fsub_rn(th[j], an[j]);
@@ -294,7 +389,7 @@ struct GpsArgs {
     float eta, beta, omb;
 };
 
-template <int UNROLL, bool STREAM>
+template <int UNROLL, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads)
 gps_kernel(const Chunk* __restrict__ chunks, GpsArgs a) {
     const Chunk c = chunks[blockIdx.x];
@@ -304,34 +399,32 @@ gps_kernel(const Chunk* __restrict__ chunks, GpsArgs a) {
     float* ib = a.inbox + c.begin;
     const float eta = a.eta, beta = a.beta, omb = a.omb;
     uint32_t done = 0;
-    if ((c.begin & 3ull) == 0) {
-        const uint32_t nvec = c.count >> 2;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
-            float4 vd[UNROLL], vx[UNROLL], vm[UNROLL];
+            FVec<VE> vd[UNROLL], vx[UNROLL], vm[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    vd[u] = ld4<STREAM>(ob + 4ull * v);
-                    vx[u] = ld4<STREAM>(Th + 4ull * v);
-                    vm[u] = ld4<STREAM>(Mg + 4ull * v);
+                    vd[u] = ldf<VE, STREAM>(ob + (size_t)VE * v);
+                    vx[u] = ldf<VE, STREAM>(Th + (size_t)VE * v);
+                    vm[u] = ldf<VE, STREAM>(Mg + (size_t)VE * v);
                 }
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    model_update(vx[u].x, vm[u].x, vd[u].x, eta, beta, omb);
-                    model_update(vx[u].y, vm[u].y, vd[u].y, eta, beta, omb);
-                    model_update(vx[u].z, vm[u].z, vd[u].z, eta, beta, omb);
-                    model_update(vx[u].w, vm[u].w, vd[u].w, eta, beta, omb);
-                    st4<STREAM>(Th + 4ull * v, vx[u]);
-                    st4<STREAM>(Mg + 4ull * v, vm[u]);
-                    st4<STREAM>(ib + 4ull * v, vx[u]);
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) model_update(vx[u].v[e], vm[u].v[e], vd[u].v[e], eta, beta, omb);
+                    stf<VE, STREAM>(Th + (size_t)VE * v, vx[u]);
+                    stf<VE, STREAM>(Mg + (size_t)VE * v, vm[u]);
+                    stf<VE, STREAM>(ib + (size_t)VE * v, vx[u]);
                 }
             }
         }
-        done = nvec << 2;
+        done = nvec * VE;
     }
     for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
         float x = Th[j], m = Mg[j];
@@ -352,7 +445,7 @@ struct PullArgs {
     float alpha, oma;
 };
 
-template <int UNROLL, bool STREAM>
+template <int UNROLL, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads)
 pull_kernel(const Chunk* __restrict__ chunks, PullArgs a) {
     const Chunk c = chunks[blockIdx.x];
@@ -361,33 +454,31 @@ pull_kernel(const Chunk* __restrict__ chunks, PullArgs a) {
     float* an = a.anchor + c.begin;
     const float alpha = a.alpha, oma = a.oma;
     uint32_t done = 0;
-    if ((c.begin & 3ull) == 0) {
-        const uint32_t nvec = c.count >> 2;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
-            float4 vx[UNROLL], vy[UNROLL];
+            FVec<VE> vx[UNROLL], vy[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    vx[u] = ld4<STREAM>(th + 4ull * v);
-                    vy[u] = ld4<STREAM>(ib + 4ull * v);
+                    vx[u] = ldf<VE, STREAM>(th + (size_t)VE * v);
+                    vy[u] = ldf<VE, STREAM>(ib + (size_t)VE * v);
                 }
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
                 if (v < nvec) {
-                    float4 r;
-                    r.x = merge(vx[u].x, vy[u].x, alpha, oma);
-                    r.y = merge(vx[u].y, vy[u].y, alpha, oma);
-                    r.z = merge(vx[u].z, vy[u].z, alpha, oma);
-                    r.w = merge(vx[u].w, vy[u].w, alpha, oma);
-                    st4<STREAM>(th + 4ull * v, r);
-                    st4<STREAM>(an + 4ull * v, r);
+                    FVec<VE> r;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) r.v[e] = merge(vx[u].v[e], vy[u].v[e], alpha, oma);
+                    stf<VE, STREAM>(th + (size_t)VE * v, r);
+                    stf<VE, STREAM>(an + (size_t)VE * v, r);
                 }
             }
         }
-        done = nvec << 2;
+        done = nvec * VE;
     }
     for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
         float r = merge(th[j], ib[j], alpha, oma);

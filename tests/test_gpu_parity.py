@@ -121,7 +121,7 @@ def test_small_shapes_bit_exact(shape, wdt, mode):
     ls.close()
 
 
-@pytest.mark.parametrize("chunk", [4, 64, 1024, 8192, 1 << 20])
+@pytest.mark.parametrize("chunk", [8, 64, 1024, 8192, 1 << 20])
 def test_chunk_size_invariance(chunk):
     lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 100000])
     worker_lps = [0, 1]
@@ -315,6 +315,7 @@ def test_config_160m_fp32_full_trace():
 
 def test_config_410m_fp32_staleness_order():
     # 32 workers with fp32 copies: ~89 GB on the device
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 100 * (1 << 30):
         pytest.skip("needs ~95 GB of free device memory")
@@ -325,3 +326,27 @@ def test_config_410m_fp32_staleness_order():
         if r["kind"] == tr.PULL:
             by_lps[r["lps"]] = by_lps.get(r["lps"], 0) + 1
     assert set(by_lps) == {0, 1, 2, 3}
+
+
+# ---------------------------------------------------------------------------------------------
+# bandwidth-sweep shapes: flat buffers and the 1.4B-class layout (the largest size), one pass of
+# every kernel, sampled outputs against the oracle
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("case,wdt", [("flat_2^24", gen.F32), ("flat_2^26", gen.BF16), ("decoder_1p4b", gen.F32)])
+def test_sweep_shapes_one_pass(case, wdt):
+    if case == "decoder_1p4b":
+        torch.cuda.empty_cache()
+        free, _ = torch.cuda.mem_get_info()
+        if free < 70 * (1 << 30):
+            pytest.skip("needs ~60 GB of free device memory")
+        lay = layouts.named_layout("1p4b")
+    else:
+        lay = layouts.flat_layout(case, 1 << int(case.split("^")[1]))
+    probes = default_probes(lay, width=8192, n_random=12, seed=1)
+    ls = Lockstep(lay, [0], dict(K=2, **PAPER_HP), wdt, seed=31, probes=probes)
+    ev = np.zeros(7, dtype=tr.EVENT_DTYPE)
+    ev["kind"] = [tr.ARRIVE, tr.ARRIVE, tr.GPS_RECV, tr.ARRIVE, tr.PULL, tr.ARRIVE, tr.ARRIVE]
+    ls.run(ev, check_every=1)
+    assert ls.bit_identical
+    assert ls.h.counters(0) == {"t": 5, "t_last": 3, "phase": hb.PUSHED, "t_push": 5, "i": 1}
+    ls.close()
