@@ -268,6 +268,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--chunk-elems", type=int, default=0)
+    ap.add_argument("--max-batch", type=int, default=1,
+                    help="multi-event fusion in the driver: up to this many arrivals per launch (1 = one kernel per event)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over buffer sizes instead of the default line")
     ap.add_argument("--sweep-max", type=int, default=0, help="largest size to include (0 = all)")
     args = ap.parse_args()
@@ -287,7 +289,7 @@ def main():
     wname = {0: "f32", 1: "bf16"}[wl.worker_dtype]
     config = {"workload": f"{wl.name}: decoder layout P={P} ({lay.n_tensors} tensors), {wl.n_workers} workers over "
                           f"{wl.n_lps} LPS, 1 GPS, fp32 master + {wname} worker copies, K={wl.K}, paper hyperparameters",
-              "events_per_step": args.events_per_step, "trace_seed": wl.seed,
+              "events_per_step": args.events_per_step, "trace_seed": wl.seed, "max_batch": args.max_batch,
               "l2": "every buffer (%.0f MB) is larger than L2; no flush needed" % (P * 4 / 1e6),
               "parallelism": "index-sharded replicas, no collective" if world > 1 else "single GPU"}
 
@@ -355,7 +357,7 @@ def main():
     def run_step(s, e2e=False, host_results=None, probe=None):
         win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
         if not e2e:
-            h.replay(win, producer_dev, want_log=False)
+            h.replay(win, producer_dev, want_log=False, max_batch=args.max_batch)
             return 0
         # end to end: results live in pinned host memory and are copied in by the library; two
         # staging buffers let the copy of the next result overlap the current update kernel
@@ -402,6 +404,7 @@ def main():
     torch.cuda.synchronize(dev)
     h.timing_enable(True)
     launches0 = h.info()["launches"]
+    batch0 = h.batch_info()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize(dev)
@@ -417,6 +420,7 @@ def main():
     elapsed_ms = e0.elapsed_time(e1)
     launches = h.info()["launches"] - launches0
     timing = h.timing_read()
+    batch1 = h.batch_info()
     h.timing_enable(False)
     units = float(args.steps * args.events_per_step) * P
     t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
@@ -424,17 +428,28 @@ def main():
 
     # ---- roofline of the dominant kernel ----
     peak, peak_kind = measured_peak_gbs()
-    n_arr, ms_arr = timing["arrive"]
-    bpp = BYTES_PER_PARAM["arrive_" + wname]
-    achieved = (bpp * P / 1e9) / (ms_arr / n_arr * 1e-3) if n_arr else None
-    tpp = DRAM_BYTES_PER_PARAM.get("arrive_" + wname)
-    traffic = tpp * P if tpp else None
-    roofline = {"bound": "hbm", "kernel": f"arrive_kernel<{wname}>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_source": f"of {peak_kind}",
-                "algorithmic_bytes_per_launch": bpp * P,
-                "per_kernel": {k: {"launches": n, "mean_ms": (ms / n if n else None),
-                                   "GBps": ((BYTES_PER_PARAM.get(k, BYTES_PER_PARAM.get(k + "_" + wname, 0)) * P / 1e9) / (ms / n * 1e-3) if n else None)}
-                               for k, (n, ms) in timing.items()}}
+    wbytes = 4 if wl.worker_dtype == gen.F32 else 2
+
+    def kernel_bytes(kind, n):
+        """algorithmic bytes of all timed launches of one kernel kind"""
+        if kind == "arrive_multi":
+            return (16 * (batch1["multi_launches"] - batch0["multi_launches"])
+                    + 3 * wbytes * (batch1["batched_arrivals"] - batch0["batched_arrivals"])) * P
+        b = BYTES_PER_PARAM.get(kind, BYTES_PER_PARAM.get(kind + "_" + wname, 0))
+        return b * P * n
+
+    per_kernel = {k: {"launches": n, "mean_ms": (ms / n if n else None), "share_of_step": ms / elapsed_ms,
+                      "GBps": (kernel_bytes(k, n) / 1e9 / (ms * 1e-3) if n else None)} for k, (n, ms) in timing.items()}
+    dominant = max(timing, key=lambda k: timing[k][1])
+    dn, dms = timing[dominant]
+    d_bytes = kernel_bytes(dominant, dn) / dn
+    achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
+    tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
+    roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": (tpp * P if tpp else None), "peak_source": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel,
+                "arrivals_per_multi_launch": ((batch1["batched_arrivals"] - batch0["batched_arrivals"])
+                                              / max(1, batch1["multi_launches"] - batch0["multi_launches"]))}
 
     # ---- end to end (host-resident worker results) ----
     e2e = None

@@ -178,6 +178,18 @@ typedef int (*halos_producer_fn)(void* user, uint32_t event_index, uint32_t work
 int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                  void* user, halos_event_log* log_host, uint32_t* failed_at);
 
+/* The same replay with multi-event fusion: up to max_batch (<= 4) arrivals at one LPS, from distinct
+ * workers, are applied by ONE kernel that reads and writes that LPS's model and momentum once for
+ * the whole batch (per element the updates are applied in queue order, so the state after the call
+ * is bit-identical to halos_replay, and so is the log except for its `fused` flags).  Counters, the
+ * log and the producer calls still follow trace order; only kernel launches are deferred, past events
+ * that touch disjoint buffers.  Consequence for the producer: a result it returned must stay valid
+ * until the producer is called again for the SAME worker or the replay returns (with halos_replay it
+ * only has to survive until the next producer call).  max_batch <= 1 behaves like halos_replay;
+ * contexts with HALOS_FLAG_STATS are never batched. */
+int halos_replay_batched(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
+                         void* user, halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch);
+
 /* Read-only device pointer to a state buffer (for inspection; valid until halos_destroy).
  * *numel = P.  Element type fp32, or worker_dtype for HALOS_BUF_THETA0. */
 int halos_peek(halos_ctx* ctx, uint32_t which, uint32_t index, const void** ptr_dev, uint64_t* numel);
@@ -201,6 +213,20 @@ int halos_stats(halos_ctx* ctx, uint32_t what, uint32_t lps, double* out_host);
 /* Number of parameters P, tensors, scheduler chunks, and kernels launched so far. */
 int halos_info(halos_ctx* ctx, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunks, uint64_t* launches);
 
+/* Checkpoint / resume.  halos_export_file writes the whole state (every buffer, all counters and
+ * phases) to a file; halos_import_file loads it into a context that was created with the same
+ * shape (P, tensors, servers, workers, worker_dtype; checked) and replaces its state, so that a
+ * replay continued after export -> destroy -> create -> import equals the uninterrupted replay bit
+ * for bit.  Both wait for the stream.  BAD_STATE if any worker result is registered but not yet
+ * applied (borrowed caller memory cannot be checkpointed); INVALID_ARG on I/O errors or a file
+ * that does not match. */
+int halos_export_file(halos_ctx* ctx, const char* path);
+int halos_import_file(halos_ctx* ctx, const char* path);
+
+/* Multi-event fusion counters since creation: launches of the multi-arrival kernel and the number
+ * of arrivals they covered (algorithmic bytes of those launches: (16 launches + 3 w_b arrivals) P). */
+int halos_batch_info(halos_ctx* ctx, uint64_t* multi_launches, uint64_t* batched_arrivals);
+
 /* Per-kernel device timing.  While enabled, every update kernel is bracketed by CUDA events on the
  * context's stream; halos_timing_read waits for the stream and returns, for one kernel kind, how
  * many launches were timed since halos_timing_enable(ctx, 1) and their summed duration. */
@@ -210,7 +236,8 @@ enum {
     HALOS_K_PUSH = 2,
     HALOS_K_GPS = 3,          /* global momentum update + Theta_i snapshot */
     HALOS_K_PULL = 4,         /* merge + anchor reset */
-    HALOS_K_COUNT = 5
+    HALOS_K_ARRIVE_MULTI = 5, /* 2-4 arrivals at one LPS in one pass (halos_replay_batched) */
+    HALOS_K_COUNT = 6
 };
 int halos_timing_enable(halos_ctx* ctx, int on);
 int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double* total_ms);

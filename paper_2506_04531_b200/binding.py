@@ -24,14 +24,15 @@ FLAG_STATS = 1
 IDLE, PUSHED, ANSWERED = 0, 1, 2
 BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0 = range(8)
 EV_ARRIVE, EV_GPS_RECV, EV_PULL = 0, 1, 2
-K_ARRIVE, K_ARRIVE_PUSH, K_PUSH, K_GPS, K_PULL = range(5)
-KERNEL_NAMES = ("arrive", "arrive_push", "push", "gps", "pull")
+K_ARRIVE, K_ARRIVE_PUSH, K_PUSH, K_GPS, K_PULL, K_ARRIVE_MULTI = range(6)
+KERNEL_NAMES = ("arrive", "arrive_push", "push", "gps", "pull", "arrive_multi")
 
 EXPORTED = (
     "halos_default_config", "halos_create", "halos_worker_delta", "halos_worker_delta_host", "halos_lps_apply",
     "halos_lps_push", "halos_gps_merge", "halos_lps_pull", "halos_destroy", "halos_replay", "halos_peek",
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
-    "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc",
+    "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
+    "halos_import_file", "halos_replay_batched", "halos_batch_info",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -95,6 +96,8 @@ def load_library():
     lib.halos_lps_pull.argtypes = [vp, u32]
     lib.halos_destroy.argtypes = [vp]
     lib.halos_replay.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32)]
+    lib.halos_replay_batched.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
+    lib.halos_batch_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
     lib.halos_peek.argtypes = [vp, u32, u32, C.POINTER(vp), C.POINTER(u64)]
     lib.halos_read.argtypes = [vp, u32, u32, u64, u64, vp]
     lib.halos_counters.argtypes = [vp, u32, vp]
@@ -103,6 +106,8 @@ def load_library():
     lib.halos_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u32), C.POINTER(u32), C.POINTER(u64)]
     lib.halos_timing_enable.argtypes = [vp, i32]
     lib.halos_timing_read.argtypes = [vp, u32, C.POINTER(u64), C.POINTER(C.c_double)]
+    lib.halos_export_file.argtypes = [vp, C.c_char_p]
+    lib.halos_import_file.argtypes = [vp, C.c_char_p]
     lib.halos_push_noalloc.argtypes = [C.c_int32, vp, vp, vp, vp, u64, vp]
     lib.halos_strerror.argtypes = [i32]
     lib.halos_strerror.restype = C.c_char_p
@@ -149,12 +154,14 @@ class Halos:
 
     ``theta_init`` is a flat fp32 CUDA tensor of P elements; ``tensor_numel`` the tensor sizes of
     the layout (defaults to one tensor of P); device memory comes from the PyTorch caching
-    allocator unless ``use_torch_allocator=False``.
+    allocator unless ``use_torch_allocator=False``; ``alloc_limit_bytes`` makes that allocator refuse
+    requests beyond a budget (used to test the out-of-memory path).
     """
 
     def __init__(self, theta_init, worker_lps: Sequence[int], tensor_numel: Optional[Sequence[int]] = None, *,
                  n_lps: Optional[int] = None, eta_l=0.2, beta_l=0.9, eta_g=0.15, beta_g=0.5, alpha=0.25, K=32,
-                 worker_dtype=F32, flags=0, chunk_elems=0, stream=None, use_torch_allocator=True):
+                 worker_dtype=F32, flags=0, chunk_elems=0, stream=None, use_torch_allocator=True,
+                 alloc_limit_bytes: Optional[int] = None):
         import torch
         self._torch = torch
         if not torch.cuda.is_available():
@@ -178,7 +185,12 @@ class Halos:
         self._blocks = {}
         self._stream = stream if stream is not None else torch.cuda.current_stream(self.device)
 
+        self._allocated = 0
+
         def _alloc(nbytes, _user):
+            if alloc_limit_bytes is not None and self._allocated + int(nbytes) > alloc_limit_bytes:
+                return None          # lets tests exercise the library's out-of-memory path
+            self._allocated += int(nbytes)
             try:
                 with torch.cuda.device(self.device):
                     t = torch.empty(int(nbytes), dtype=torch.uint8, device=self.device)
@@ -263,9 +275,11 @@ class Halos:
         self._check(self._lib.halos_lps_pull(self._h, lps))
 
     # ------------------------------------------------------------------ auxiliary
-    def replay(self, events: np.ndarray, producer: Callable, want_log: bool = True):
+    def replay(self, events: np.ndarray, producer: Callable, want_log: bool = True, max_batch: int = 1):
         """events: structured array (kind, lps, worker, pad, time_ns); producer(event_index, worker, round)
-        returns a flat tensor/address or a list of per-tensor tensors.  Returns the event log."""
+        returns a flat tensor/address or a list of per-tensor tensors.  max_batch > 1 turns on multi-event
+        fusion (then a result must stay valid until the producer is called again for the same worker).
+        Returns the event log."""
         ev = np.ascontiguousarray(events)
         assert ev.dtype.itemsize == C.sizeof(Event)
         log = np.zeros(len(ev), dtype=EVENT_LOG_DTYPE) if want_log else None
@@ -277,7 +291,7 @@ class Halos:
                 r = producer(int(index), int(worker), int(rnd))
                 if isinstance(r, (list, tuple)):
                     arr = (C.c_void_p * self.n_tensors)(*[_ptr(t) for t in r])
-                    hold[worker] = (r, arr)
+                    hold[(worker, "p")] = (r, arr)
                     ptrs_out[0] = C.cast(arr, C.POINTER(C.c_void_p))
                 else:
                     hold[worker] = r
@@ -289,8 +303,8 @@ class Halos:
 
         cb = PRODUCER_FN(_prod)
         failed = C.c_uint32(0)
-        rc = self._lib.halos_replay(self._h, ev.ctypes.data, len(ev), cb, None,
-                                    log.ctypes.data if log is not None else None, C.byref(failed))
+        rc = self._lib.halos_replay_batched(self._h, ev.ctypes.data, len(ev), cb, None,
+                                            log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch))
         if err:
             raise err[0]
         if rc != OK:
@@ -335,6 +349,17 @@ class Halos:
         P, nt, nc, nl = C.c_uint64(), C.c_uint32(), C.c_uint32(), C.c_uint64()
         self._check(self._lib.halos_info(self._h, C.byref(P), C.byref(nt), C.byref(nc), C.byref(nl)))
         return {"P": P.value, "n_tensors": nt.value, "n_chunks": nc.value, "launches": nl.value}
+
+    def export_file(self, path):
+        self._check(self._lib.halos_export_file(self._h, str(path).encode()))
+
+    def import_file(self, path):
+        self._check(self._lib.halos_import_file(self._h, str(path).encode()))
+
+    def batch_info(self) -> dict:
+        a, b = C.c_uint64(), C.c_uint64()
+        self._check(self._lib.halos_batch_info(self._h, C.byref(a), C.byref(b)))
+        return {"multi_launches": a.value, "batched_arrivals": b.value}
 
     def timing_enable(self, on: bool = True):
         self._check(self._lib.halos_timing_enable(self._h, int(on)))

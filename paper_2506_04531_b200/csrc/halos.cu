@@ -81,6 +81,8 @@ struct halos_ctx {
 
     std::vector<void*> owned;  // device allocations made through the allocator
     uint64_t launches = 0;
+    uint64_t batched_arrivals = 0;  // arrivals that ran inside a multi-arrival launch
+    uint64_t multi_launches = 0;
     bool timing = false;
     std::vector<TimedLaunch> timed;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
@@ -238,34 +240,23 @@ int finalize_stats(halos_ctx* c, uint32_t what, uint32_t lps) {
     return HALOS_OK;
 }
 
-// lps_apply with an optional fused push; shared by the C entry point and the replay driver.
-int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int* push_due) {
+// Host-side part of an arrival (Alg. 1 lines 10 and 13): argument/state checks and counter updates.
+// *due = this arrival completes a window of K; *push = the caller wants Delta formed with it.
+int apply_check(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, bool* due, bool* push) {
     if (lps >= c->cfg.n_lps || worker >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "lps/worker out of range");
     WorkerState& w = c->workers[worker];
     if (w.lps != lps) return fail(c, HALOS_ERR_INVALID_ARG, "worker %u does not belong to LPS %u", worker, lps);
     if (w.pending == PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u has no pending result", worker);
     LpsState& s = c->lps[lps];
-    const bool due = (s.t + 1 - s.t_last == c->cfg.K);
-    const bool push = fuse_push && due;
-    if (push && s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u: push due while a round trip is in flight", lps);
-    CU(c, cudaSetDevice(c->cfg.device));
-    const void* flat = nullptr;
-    if (w.pending == PEND_FLAT) flat = w.flat;
-    if (w.pending == PEND_STAGED) {
-        flat = c->stage[w.slot];
-        CU(c, cudaStreamWaitEvent(c->stream, c->stage_ready[w.slot], 0));
-    }
-    int rc = c->wb == 4 ? launch_arrive<float>(c, s, w, worker, push, flat)
-                        : launch_arrive<uint16_t>(c, s, w, worker, push, flat);
-    if (rc != HALOS_OK) return rc;
-    if (w.pending == PEND_STAGED) {
-        CU(c, cudaEventRecord(c->stage_free[w.slot], c->stream));
-        c->stage_owner[w.slot] = -1;
-    }
-    if (c->cfg.flags & HALOS_FLAG_STATS) {
-        if ((rc = finalize_stats(c, 0, lps)) != HALOS_OK) return rc;
-        if (push && (rc = finalize_stats(c, 1, lps)) != HALOS_OK) return rc;
-    }
+    *due = (s.t + 1 - s.t_last == c->cfg.K);
+    *push = fuse_push && *due;
+    if (*push && s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u: push due while a round trip is in flight", lps);
+    return HALOS_OK;
+}
+
+void apply_commit(halos_ctx* c, uint32_t lps, uint32_t worker, bool push) {
+    WorkerState& w = c->workers[worker];
+    LpsState& s = c->lps[lps];
     w.pending = PEND_NONE;
     w.flat = nullptr;
     w.slot = -1;
@@ -276,8 +267,93 @@ int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int*
         s.phase = HALOS_PUSHED;
         s.t_push = s.t;
     }
+}
+
+// lps_apply with an optional fused push; shared by the C entry point and the replay driver.
+int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int* push_due) {
+    bool due = false, push = false;
+    int rc = apply_check(c, lps, worker, fuse_push, &due, &push);
+    if (rc != HALOS_OK) return rc;
+    WorkerState& w = c->workers[worker];
+    LpsState& s = c->lps[lps];
+    CU(c, cudaSetDevice(c->cfg.device));
+    const void* flat = nullptr;
+    if (w.pending == PEND_FLAT) flat = w.flat;
+    if (w.pending == PEND_STAGED) {
+        flat = c->stage[w.slot];
+        CU(c, cudaStreamWaitEvent(c->stream, c->stage_ready[w.slot], 0));
+    }
+    rc = c->wb == 4 ? launch_arrive<float>(c, s, w, worker, push, flat)
+                    : launch_arrive<uint16_t>(c, s, w, worker, push, flat);
+    if (rc != HALOS_OK) return rc;
+    if (w.pending == PEND_STAGED) {
+        CU(c, cudaEventRecord(c->stage_free[w.slot], c->stream));
+        c->stage_owner[w.slot] = -1;
+    }
+    if (c->cfg.flags & HALOS_FLAG_STATS) {
+        if ((rc = finalize_stats(c, 0, lps)) != HALOS_OK) return rc;
+        if (push && (rc = finalize_stats(c, 1, lps)) != HALOS_OK) return rc;
+    }
+    apply_commit(c, lps, worker, push);
     if (push_due) *push_due = due ? 1 : 0;
     return HALOS_OK;
+}
+
+// ---- batched arrivals (multi-event fusion) -------------------------------------------------------
+struct Deferred {
+    uint32_t worker;
+    const void* flat;   // NULL: per-tensor pointer table of that worker
+};
+
+template <class W, int NB>
+int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push) {
+    ArriveMultiArgs<W> a;
+    const size_t nt = c->tensor_numel.size();
+    for (int j = 0; j < kMaxBatch; ++j) {
+        const int k = j < NB ? j : 0;
+        a.h_flat[j] = (const W*)d[k].flat;
+        a.h_ptrs[j] = d[k].flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)d[k].worker * nt);
+        a.th0[j] = (W*)c->workers[d[k].worker].th0;
+    }
+    a.tensor_off = c->d_tensor_off;
+    a.th = s.th;
+    a.ml = s.ml;
+    a.anchor = s.anchor;
+    a.outbox = s.outbox;
+    a.eta = c->cfg.eta_l;
+    a.beta = c->cfg.beta_l;
+    a.omb = 1.0f - c->cfg.beta_l;
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    Timer tm(c, HALOS_K_ARRIVE_MULTI);
+    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    else arrive_multi_kernel<W, NB, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    tm.stop();
+    c->launches++;
+    c->batched_arrivals += NB;
+    c->multi_launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+
+template <class W>
+int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool push) {
+    LpsState& s = c->lps[lps];
+    if (q.empty()) return HALOS_OK;
+    int rc = HALOS_OK;
+    CU(c, cudaSetDevice(c->cfg.device));
+    switch (q.size()) {
+        case 1: rc = launch_arrive<W>(c, s, c->workers[q[0].worker], q[0].worker, push, q[0].flat); break;
+        case 2: rc = launch_arrive_multi<W, 2>(c, s, q.data(), push); break;
+        case 3: rc = launch_arrive_multi<W, 3>(c, s, q.data(), push); break;
+        case 4: rc = launch_arrive_multi<W, 4>(c, s, q.data(), push); break;
+        default: rc = fail(c, HALOS_ERR_INVALID_ARG, "internal: batch larger than %d", kMaxBatch);
+    }
+    q.clear();
+    return rc;
+}
+
+int flush_deferred(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool push) {
+    return c->wb == 4 ? flush_deferred_t<float>(c, lps, q, push) : flush_deferred_t<uint16_t>(c, lps, q, push);
 }
 
 }  // namespace
@@ -557,13 +633,26 @@ int halos_lps_pull(halos_ctx* c, uint32_t lps) {
 }
 
 // ------------------------------------------------------------------------------ event-queue driver
-int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
-                 halos_event_log* log, uint32_t* failed_at) {
+// Events are taken in trace order: counters, phases, the log and the producer calls follow that order
+// exactly.  With max_batch > 1 the LAUNCH of an arrival may be deferred: arrivals at one LPS wait in
+// that LPS's queue and are flushed as one multi-arrival launch when the queue is full, when the same
+// worker arrives again, when the arrival closes a window of K (it is flushed with the push fused), when
+// a PULL for that LPS comes up, or at the end.  Everything an arrival at LPS l touches (theta_l, m_l,
+// the worker's snapshot; outbox_l only when it pushes) is disjoint from what events of other LPSs and
+// GPS_RECV(l) touch, so the deferred launches commute with the launches they are moved past and the
+// final state is bit-identical to the unbatched replay.
+int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
+                         halos_event_log* log, uint32_t* failed_at, uint32_t max_batch) {
     if (!c) return HALOS_ERR_INVALID_ARG;
     if (n && !ev) return fail(c, HALOS_ERR_INVALID_ARG, "null event array");
-    for (uint32_t k = 0; k < n; ++k) {
+    if (max_batch == 0) max_batch = 1;
+    if (max_batch > (uint32_t)kMaxBatch) max_batch = kMaxBatch;
+    if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
+    std::vector<std::vector<Deferred>> queue(c->cfg.n_lps);
+    int rc = HALOS_OK;
+    uint32_t k = 0;
+    for (; k < n && rc == HALOS_OK; ++k) {
         const halos_event& e = ev[k];
-        int rc = HALOS_OK;
         halos_event_log rec;
         std::memset(&rec, 0, sizeof rec);
         rec.index = k;
@@ -572,46 +661,169 @@ int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer
         rec.worker = e.worker;
         if (e.lps >= c->cfg.n_lps) rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: lps out of range", k);
         else if (e.kind == HALOS_EV_ARRIVE) {
+            std::vector<Deferred>& q = queue[e.lps];
             if (e.worker >= c->cfg.n_workers) rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: worker out of range", k);
-            else if (!producer) rc = fail(c, HALOS_ERR_INVALID_ARG, "ARRIVE events need a producer");
+            else if (!producer && c->workers[e.worker].pending == PEND_NONE) rc = fail(c, HALOS_ERR_INVALID_ARG, "ARRIVE events need a producer");
             else {
                 WorkerState& w = c->workers[e.worker];
+                for (const Deferred& d : q)
+                    if (d.worker == e.worker) {   // its previous result is still queued: run it first
+                        rc = flush_deferred(c, e.lps, q, false);
+                        break;
+                    }
                 const void* flat = nullptr;
                 const void* const* ptrs = nullptr;
-                if (w.pending == PEND_NONE) {
+                if (rc == HALOS_OK && w.pending == PEND_NONE) {
                     if (producer(user, k, e.worker, w.round, &flat, &ptrs) != 0)
                         rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: producer failed", k);
                     else rc = halos_worker_delta(c, e.worker, flat, ptrs);
                 }
+                bool due = false, push = false;
+                if (rc == HALOS_OK) rc = apply_check(c, e.lps, e.worker, true, &due, &push);
+                if (rc == HALOS_OK && w.pending == PEND_STAGED && !q.empty()) rc = flush_deferred(c, e.lps, q, false);
                 if (rc == HALOS_OK) {
                     rec.worker_staleness = c->lps[e.lps].t - w.sched_t;
-                    int due = 0;
-                    rc = apply_impl(c, e.lps, e.worker, true, &due);
-                    rec.pushed = (uint8_t)due;
-                    rec.fused = (uint8_t)due;
+                    if (w.pending == PEND_STAGED) {
+                        rc = apply_impl(c, e.lps, e.worker, true, nullptr);   // host-staged results are not deferred
+                    } else {
+                        q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr});
+                        rec.fused = (uint8_t)(q.size() > 1 || push);
+                        apply_commit(c, e.lps, e.worker, push);
+                        if (push || q.size() >= max_batch) rc = flush_deferred(c, e.lps, q, push);
+                    }
+                    rec.pushed = (uint8_t)push;
                 }
             }
         } else if (e.kind == HALOS_EV_GPS_RECV) {
             rc = halos_gps_merge(c, e.lps);
         } else if (e.kind == HALOS_EV_PULL) {
-            if (c->lps[e.lps].phase == HALOS_ANSWERED) rec.gps_lag = c->gps_iter - c->lps[e.lps].inbox_iter;
-            rc = halos_lps_pull(c, e.lps);
+            rc = flush_deferred(c, e.lps, queue[e.lps], false);
+            if (rc == HALOS_OK) {
+                if (c->lps[e.lps].phase == HALOS_ANSWERED) rec.gps_lag = c->gps_iter - c->lps[e.lps].inbox_iter;
+                rc = halos_lps_pull(c, e.lps);
+            }
         } else {
             rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: unknown kind %u", k, (unsigned)e.kind);
         }
-        if (rc != HALOS_OK) {
-            if (failed_at) *failed_at = k;
-            return rc;
-        }
-        if (log) {
+        if (rc == HALOS_OK && log) {
             rec.t = c->lps[e.lps].t;
             rec.t_last = c->lps[e.lps].t_last;
             rec.gps_iter = c->gps_iter;
             log[k] = rec;
         }
     }
+    // whatever is still queued belongs to events already accounted for: launch it
+    for (uint32_t l = 0; l < c->cfg.n_lps; ++l) {
+        int rf = flush_deferred(c, l, queue[l], false);
+        if (rc == HALOS_OK && rf != HALOS_OK) rc = rf;
+    }
+    if (rc != HALOS_OK && failed_at) *failed_at = k ? k - 1 : 0;
+    return rc;
+}
+
+int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
+                 halos_event_log* log, uint32_t* failed_at) {
+    return halos_replay_batched(c, ev, n, producer, user, log, failed_at, 1);
+}
+
+// ------------------------------------------------------------------------------ checkpoint / resume
+namespace {
+struct CkptHeader {
+    char magic[8];
+    uint32_t version, wb;
+    uint64_t P;
+    uint32_t n_lps, n_workers, n_tensors, K;
+    float eta_l, beta_l, eta_g, beta_g, alpha;
+    uint32_t pad;
+    uint64_t gps_iter;
+};
+struct CkptLps { uint64_t t, t_last, t_push, inbox_iter; int32_t phase; int32_t pad; };
+struct CkptWorker { uint64_t round, sched_t; };
+constexpr size_t kBounce = 64u << 20;
+
+int stream_buffer(halos_ctx* c, FILE* f, void* dev, size_t bytes, bool to_file, void* bounce) {
+    for (size_t off = 0; off < bytes; off += kBounce) {
+        const size_t n = bytes - off < kBounce ? bytes - off : kBounce;
+        if (to_file) {
+            CU(c, cudaMemcpyAsync(bounce, (char*)dev + off, n, cudaMemcpyDeviceToHost, c->stream));
+            CU(c, cudaStreamSynchronize(c->stream));
+            if (fwrite(bounce, 1, n, f) != n) return fail(c, HALOS_ERR_INVALID_ARG, "short write to checkpoint file");
+        } else {
+            if (fread(bounce, 1, n, f) != n) return fail(c, HALOS_ERR_INVALID_ARG, "checkpoint file is truncated");
+            CU(c, cudaMemcpyAsync((char*)dev + off, bounce, n, cudaMemcpyHostToDevice, c->stream));
+            CU(c, cudaStreamSynchronize(c->stream));
+        }
+    }
     return HALOS_OK;
 }
+
+int checkpoint(halos_ctx* c, const char* path, bool to_file) {
+    if (!c || !path) return HALOS_ERR_INVALID_ARG;
+    for (auto& w : c->workers)
+        if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "a worker result is registered but not applied");
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->stream));
+    FILE* f = fopen(path, to_file ? "wb" : "rb");
+    if (!f) return fail(c, HALOS_ERR_INVALID_ARG, "cannot open %s", path);
+    void* bounce = nullptr;
+    if (cudaHostAlloc(&bounce, kBounce, cudaHostAllocDefault) != cudaSuccess) {
+        (void)cudaGetLastError();
+        fclose(f);
+        return fail(c, HALOS_ERR_OOM, "pinned bounce buffer allocation failed");
+    }
+    int rc = HALOS_OK;
+    CkptHeader h;
+    std::memset(&h, 0, sizeof h);
+    std::vector<CkptLps> ls(c->lps.size());
+    std::vector<CkptWorker> ws(c->workers.size());
+    if (to_file) {
+        std::memcpy(h.magic, "HALOSCK1", 8);
+        h.version = 1; h.wb = c->wb; h.P = c->P;
+        h.n_lps = c->cfg.n_lps; h.n_workers = c->cfg.n_workers; h.n_tensors = c->cfg.n_tensors; h.K = c->cfg.K;
+        h.eta_l = c->cfg.eta_l; h.beta_l = c->cfg.beta_l; h.eta_g = c->cfg.eta_g; h.beta_g = c->cfg.beta_g; h.alpha = c->cfg.alpha;
+        h.gps_iter = c->gps_iter;
+        for (size_t l = 0; l < ls.size(); ++l)
+            ls[l] = CkptLps{c->lps[l].t, c->lps[l].t_last, c->lps[l].t_push, c->lps[l].inbox_iter, c->lps[l].phase, 0};
+        for (size_t w = 0; w < ws.size(); ++w) ws[w] = CkptWorker{c->workers[w].round, c->workers[w].sched_t};
+        if (fwrite(&h, sizeof h, 1, f) != 1 || fwrite(c->tensor_numel.data(), 8, c->tensor_numel.size(), f) != c->tensor_numel.size() ||
+            fwrite(ls.data(), sizeof(CkptLps), ls.size(), f) != ls.size() || fwrite(ws.data(), sizeof(CkptWorker), ws.size(), f) != ws.size())
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "short write to checkpoint file");
+    } else {
+        std::vector<uint64_t> numel(c->tensor_numel.size());
+        if (fread(&h, sizeof h, 1, f) != 1 || std::memcmp(h.magic, "HALOSCK1", 8) != 0 || h.version != 1)
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "not a checkpoint file of this library");
+        else if (h.P != c->P || h.wb != c->wb || h.n_lps != c->cfg.n_lps || h.n_workers != c->cfg.n_workers || h.n_tensors != c->cfg.n_tensors)
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint shape does not match this context");
+        else if (fread(numel.data(), 8, numel.size(), f) != numel.size() || numel != c->tensor_numel)
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint tensor sizes do not match this context");
+        else if (fread(ls.data(), sizeof(CkptLps), ls.size(), f) != ls.size() || fread(ws.data(), sizeof(CkptWorker), ws.size(), f) != ws.size())
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint file is truncated");
+    }
+    auto pass = [&](void* dev, size_t bytes) {
+        if (rc == HALOS_OK) rc = stream_buffer(c, f, dev, bytes, to_file, bounce);
+    };
+    pass(c->Theta, c->P * 4);
+    pass(c->Mg, c->P * 4);
+    for (auto& s : c->lps) {
+        pass(s.th, c->P * 4); pass(s.ml, c->P * 4); pass(s.anchor, c->P * 4); pass(s.outbox, c->P * 4); pass(s.inbox, c->P * 4);
+    }
+    for (auto& w : c->workers) pass(w.th0, c->P * c->wb);
+    if (rc == HALOS_OK && !to_file) {
+        c->gps_iter = h.gps_iter;
+        for (size_t l = 0; l < ls.size(); ++l) {
+            c->lps[l].t = ls[l].t; c->lps[l].t_last = ls[l].t_last; c->lps[l].t_push = ls[l].t_push;
+            c->lps[l].inbox_iter = ls[l].inbox_iter; c->lps[l].phase = ls[l].phase;
+        }
+        for (size_t w = 0; w < ws.size(); ++w) { c->workers[w].round = ws[w].round; c->workers[w].sched_t = ws[w].sched_t; }
+    }
+    cudaFreeHost(bounce);
+    if (fclose(f) != 0 && rc == HALOS_OK && to_file) rc = fail(c, HALOS_ERR_INVALID_ARG, "closing the checkpoint file failed");
+    return rc;
+}
+}  // namespace
+
+int halos_export_file(halos_ctx* c, const char* path) { return checkpoint(c, path, true); }
+int halos_import_file(halos_ctx* c, const char* path) { return checkpoint(c, path, false); }
 
 // ------------------------------------------------------------------------------ inspection
 static int buffer_of(halos_ctx* c, uint32_t which, uint32_t index, const void** p, uint32_t* elem_bytes) {
@@ -698,6 +910,13 @@ int halos_info(halos_ctx* c, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunk
     if (n_tensors) *n_tensors = (uint32_t)c->tensor_numel.size();
     if (n_chunks) *n_chunks = (uint32_t)c->chunks.size();
     if (launches) *launches = c->launches;
+    return HALOS_OK;
+}
+
+int halos_batch_info(halos_ctx* c, uint64_t* multi_launches, uint64_t* batched_arrivals) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (multi_launches) *multi_launches = c->multi_launches;
+    if (batched_arrivals) *batched_arrivals = c->batched_arrivals;
     return HALOS_OK;
 }
 

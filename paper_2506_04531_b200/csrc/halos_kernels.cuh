@@ -322,6 +322,95 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
 }
 
 // =====================================================================================================
+// ARRIVE x NB: NB consecutive arrivals at the same LPS (distinct workers) in ONE pass.  The LPS model
+// and momentum are read and written once for the whole batch; per element the NB updates are applied
+// in queue order in registers, so the result is bit-identical to NB single launches.  Traffic per
+// batch: 8 + 8 (theta, m read + write) + NB x (2 w_b read + w_b write) instead of NB x (16 + 3 w_b).
+// Only the last arrival of a batch may close a window of K (PUSH).
+// =====================================================================================================
+constexpr int kMaxBatch = 4;
+
+template <class W>
+struct ArriveMultiArgs {
+    const W* h_flat[kMaxBatch];          // per arrival: flat result ...
+    const W* const* h_ptrs[kMaxBatch];   // ... or per-tensor pointer table
+    W* th0[kMaxBatch];                   // per arrival: that worker's start snapshot
+    const unsigned long long* tensor_off;
+    float* th;
+    float* ml;
+    const float* anchor;
+    float* outbox;
+    float eta, beta, omb;
+};
+
+template <class W, int NB, bool PUSH, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, (NB <= 2 ? 1024 / kThreads : 1))
+arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
+    using T = WTraits<W>;
+    const Chunk c = chunks[blockIdx.x];
+    const W* h[NB];
+    W* s0[NB];
+    bool vec_ok = (c.begin % VE) == 0;
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        h[j] = a.h_flat[j] ? a.h_flat[j] + c.begin : a.h_ptrs[j][c.tensor] + (c.begin - a.tensor_off[c.tensor]);
+        s0[j] = a.th0[j] + c.begin;
+        vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(h[j]) % (VE * sizeof(W))) == 0);
+    }
+    float* th = a.th + c.begin;
+    float* ml = a.ml + c.begin;
+    const float* an = PUSH ? a.anchor + c.begin : nullptr;
+    float* ob = PUSH ? a.outbox + c.begin : nullptr;
+    const float eta = a.eta, beta = a.beta, omb = a.omb;
+    uint32_t done = 0;
+    if (vec_ok) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vh[NB], vs[NB], vx, vm, va;
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                vh[j] = T::template load<VE, STREAM>(h[j] + o);
+                vs[j] = T::template load<VE, STREAM>(s0[j] + o);
+            }
+            vx = ldf<VE, STREAM>(th + o);
+            vm = ldf<VE, STREAM>(ml + o);
+            if (PUSH) va = ldf<VE, STREAM>(an + o);
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+#pragma unroll
+                for (int e = 0; e < VE; ++e) {
+                    const float d = __fsub_rn(vh[j].v[e], vs[j].v[e]);
+                    model_update(vx.v[e], vm.v[e], d, eta, beta, omb);
+                }
+                T::template store<VE, STREAM>(s0[j] + o, vx);   // worker j restarts from the model after ITS update
+            }
+            stf<VE, STREAM>(th + o, vx);
+            stf<VE, STREAM>(ml + o, vm);
+            if (PUSH) {
+                FVec<VE> D;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                stf<VE, STREAM>(ob + o, D);
+            }
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t i = done + threadIdx.x; i < c.count; i += kThreads) {
+        float x = th[i], m = ml[i];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
+            model_update(x, m, d, eta, beta, omb);
+            T::store1(s0[j] + i, x);
+        }
+        th[i] = x;
+        ml[i] = m;
+        if (PUSH) ob[i] = __fsub_rn(x, an[i]);
+    }
+}
+
+// =====================================================================================================
 // PUSH alone: Delta = theta_t - theta_{t_last}                                   Alg. 1 line 14
 // =====================================================================================================
 struct PushArgs {

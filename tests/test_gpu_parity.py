@@ -350,3 +350,153 @@ def test_sweep_shapes_one_pass(case, wdt):
     assert ls.bit_identical
     assert ls.h.counters(0) == {"t": 5, "t_last": 3, "phase": hb.PUSHED, "t_push": 5, "i": 1}
     ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# checkpoint / resume and the out-of-memory path (failures are made on the host)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+def test_checkpoint_resume_is_bit_identical(tmp_path, wdt):
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.decoder_layout("tiny", 2, 64, 300)
+    worker_lps = [0, 0, 1, 1]
+    hp = dict(K=4, **PAPER_HP)
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=[1.0, 2.5, 3.0, 1.7],
+                                            t_profiled_ms=1.0, n_arrivals=90, K=4))
+    cut = 41
+    assert any(int(e["kind"]) == tr.PULL for e in events[cut:]) and any(int(e["kind"]) == tr.GPS_RECV for e in events[:cut])
+    dg = DeviceGenerator(lay, 17)
+    scratch = torch.empty(lay.P, dtype=torch.float32 if wdt == gen.F32 else torch.int16, device="cuda")
+
+    def run(h, evs):
+        def producer(index, worker, rnd):
+            return dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=scratch, worker_dtype=wdt)
+        return h.replay(evs, producer)
+
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, **hp)
+    log_ref = run(ref, events)
+    a = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, **hp)
+    run(a, events[:cut])
+    path = tmp_path / "state.ckpt"
+    a.export_file(path)
+    counters = [a.counters(l) for l in (0, 1)]
+    a.close()
+    b = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, worker_dtype=wdt, **hp)
+    b.import_file(path)
+    assert [b.counters(l) for l in (0, 1)] == counters
+    log_b = run(b, events[cut:])
+    for which in range(8):
+        n = len(worker_lps) if which == hb.BUF_THETA0 else (1 if which < 2 else 2)
+        for idx in range(n):
+            assert np.array_equal(ref.read(which, idx).view(np.uint8), b.read(which, idx).view(np.uint8)), (which, idx)
+    for f in ("t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+        assert np.array_equal(log_ref[f][cut:], log_b[f])
+    # a file of another shape is refused and leaves the state alone
+    other = hb.Halos(torch.zeros(64, device="cuda"), [0])
+    with pytest.raises(hb.HalosError) as e:
+        other.import_file(path)
+    assert e.value.status == hb.ERR_INVALID_ARG
+    # pending results cannot be checkpointed
+    b.worker_delta(0, scratch)
+    with pytest.raises(hb.HalosError) as e:
+        b.export_file(tmp_path / "x.ckpt")
+    assert e.value.status == hb.ERR_BAD_STATE
+    for h in (ref, b, other):
+        h.close()
+
+
+def test_out_of_memory_is_reported_and_cleaned_up():
+    P = 1 << 16
+    init = torch.zeros(P, device="cuda")
+    need = P * 4 * (2 + 5 * 2 + 3)
+    for budget in (1024, P * 4 * 3, need - 1):
+        with pytest.raises(hb.HalosError) as e:
+            hb.Halos(init, [0, 1, 1], alloc_limit_bytes=budget)
+        assert e.value.status == hb.ERR_OOM
+    h = hb.Halos(init, [0, 1, 1], alloc_limit_bytes=need + (1 << 20))
+    assert h.counters(1)["t"] == 0
+    # the staging buffer for host-resident results does not fit in the budget: reported, state unchanged
+    host = torch.zeros(P).pin_memory()
+    h2 = hb.Halos(init, [0], alloc_limit_bytes=P * 4 * 8 + 65536)
+    with pytest.raises(hb.HalosError) as e:
+        h2.worker_delta_host(0, host)
+    assert e.value.status == hb.ERR_OOM and h2.worker_info(0)["pending"] is False
+    h.close()
+    h2.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# multi-event fusion: batched replay leaves exactly the state and the log of the unbatched replay
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+@pytest.mark.parametrize("mode", ["flat", "ptrs"])
+@pytest.mark.parametrize("max_batch", [2, 3, 4, 9])
+def test_batched_replay_is_bit_identical(wdt, mode, max_batch):
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 3])
+    worker_lps = [0, 0, 0, 0, 0, 1, 1, 1, 2]
+    hp = dict(K=5, **PAPER_HP)
+    speeds = [1.0, 2.5, 3.0, 1.7, 3.9, 1.1, 1.2, 3.3, 2.0]
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=speeds, t_profiled_ms=1.0,
+                                            n_arrivals=260, K=5))
+    dg = DeviceGenerator(lay, 23)
+    tdt = torch.float32 if wdt == gen.F32 else torch.int16
+    off = lay.offsets.astype(np.int64)
+
+    def make(h):
+        # one result buffer per worker: with batching a result must survive until that worker's next call
+        bufs = [torch.empty(lay.P, dtype=tdt, device="cuda") for _ in worker_lps]
+
+        def producer(index, worker, rnd):
+            r = dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker], worker_dtype=wdt)
+            if mode == "flat":
+                return r
+            return [r[off[k]:off[k + 1]] for k in range(lay.n_tensors)]
+        return producer
+
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, chunk_elems=1024, **hp)
+    log_ref = ref.replay(events, make(ref))
+    bat = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, chunk_elems=1024, **hp)
+    bat.timing_enable(True)
+    log_bat = bat.replay(events, make(bat), max_batch=max_batch)
+    timing = bat.timing_read()
+    assert timing["arrive_multi"][0] > 10                      # batches did form
+    assert bat.info()["launches"] < ref.info()["launches"]
+    for which in range(8):
+        n = len(worker_lps) if which == hb.BUF_THETA0 else (1 if which < 2 else 3)
+        for idx in range(n):
+            assert np.array_equal(ref.read(which, idx).view(np.uint8), bat.read(which, idx).view(np.uint8)), (which, idx)
+    for f in ("index", "kind", "lps", "worker", "t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+        assert np.array_equal(log_ref[f], log_bat[f]), f
+    for l in range(3):
+        assert ref.counters(l) == bat.counters(l)
+    ref.close()
+    bat.close()
+
+
+def test_batched_replay_against_oracle_160m_window():
+    """Full-size buffers, batched driver, oracle on probe windows (first 300 events of the 160m trace)."""
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    wl = workloads.workload("160m")
+    lay = wl.layout
+    probes = default_probes(lay, width=4096, n_random=6, seed=9)
+    events = wl.trace()[:300]
+    ls = Lockstep(lay, wl.worker_lps, wl.hyper(), wl.worker_dtype, wl.seed, probes=probes)
+    bufs = [torch.empty(lay.P, dtype=torch.float32, device="cuda") for _ in range(wl.n_workers)]
+
+    def producer(index, worker, rnd):
+        return ls.dgen.worker_result(ls.h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker])
+
+    ls.h.replay(events, producer, max_batch=4)
+    # the oracle side of the lock-step harness, event by event
+    for ev in events:
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        if kind == tr.ARRIVE:
+            ls.o.arrive(w, ls._oracle_result(w, ls.o.worker_info(w)["round"]))
+        elif kind == tr.GPS_RECV:
+            ls.o.gps_recv(l)
+        else:
+            ls.o.pull(l)
+    ls.compare(ls.all_buffers(), FULL_TRACE_TOL)
+    assert ls.bit_identical
+    ls.close()
