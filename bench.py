@@ -8,7 +8,9 @@ updates, merges) of the workload's seeded asynchronous trace through the library
 driver: one fused kernel per event over all tensors of the model.  Metric: parameters updated per
 second (every event updates the P parameters of one model).
 
-    value       device-resident: each worker's result theta_H already sits in HBM
+    value       device-resident: each worker's result theta_H already sits in HBM; the driver fuses up to
+                --max-batch arrivals at one LPS into one launch (bit-identical to one launch per
+                event, which is measured too and reported under per_event_kernels)
     e2e         the same replay through the C ABI with HOST-resident worker results (pinned), the
                 host->device copy of every result and a device->host read of a probe of the
                 models inside the timed region
@@ -268,7 +270,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--chunk-elems", type=int, default=0)
-    ap.add_argument("--max-batch", type=int, default=1,
+    ap.add_argument("--max-batch", type=int, default=4,
                     help="multi-event fusion in the driver: up to this many arrivals per launch (1 = one kernel per event)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over buffer sizes instead of the default line")
     ap.add_argument("--sweep-max", type=int, default=0, help="largest size to include (0 = all)")
@@ -339,7 +341,7 @@ def main():
     from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
 
     n_steps = args.steps + args.warmup
-    events = window_events(n_steps * (1 if args.no_e2e else 2), args.events_per_step, wl)
+    events = window_events(n_steps * 2 + 8, args.events_per_step, wl)
     seed = wl.seed + 1000 * rank                      # each rank: its own shard of a larger model
     dgen = DeviceGenerator(lay, seed, device=dev)
     init = dgen.theta_init()
@@ -356,9 +358,6 @@ def main():
 
     def run_step(s, e2e=False, host_results=None, probe=None):
         win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
-        if not e2e:
-            h.replay(win, producer_dev, want_log=False, max_batch=args.max_batch)
-            return 0
         # end to end: results live in pinned host memory and are copied in by the library; two
         # staging buffers let the copy of the next result overlap the current update kernel
         from paper_2506_04531_b200.inputs import trace as tr
@@ -398,58 +397,69 @@ def main():
             got += h.read(which, idx, 0, 1024).nbytes
         return got
 
-    # ---- warm-up, then the timed region (device-resident) ----
-    for s in range(args.warmup):
-        run_step(s)
-    torch.cuda.synchronize(dev)
-    h.timing_enable(True)
-    launches0 = h.info()["launches"]
-    batch0 = h.batch_info()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize(dev)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local_rank) as clk:
-        e0.record()
-        for s in range(args.warmup, n_steps):
-            run_step(s)
-        e1.record()
-        torch.cuda.synchronize(dev)
-    if world > 1:
-        dist.barrier()
-    elapsed_ms = e0.elapsed_time(e1)
-    launches = h.info()["launches"] - launches0
-    timing = h.timing_read()
-    batch1 = h.batch_info()
-    h.timing_enable(False)
-    units = float(args.steps * args.events_per_step) * P
-    t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
-    value = units_all / (t_ms * 1e-3)
-
-    # ---- roofline of the dominant kernel ----
+    # ---- warm-up, then the timed region (device-resident); once per driver mode ----
     peak, peak_kind = measured_peak_gbs()
     wbytes = 4 if wl.worker_dtype == gen.F32 else 2
 
-    def kernel_bytes(kind, n):
-        """algorithmic bytes of all timed launches of one kernel kind"""
-        if kind == "arrive_multi":
-            return (16 * (batch1["multi_launches"] - batch0["multi_launches"])
-                    + 3 * wbytes * (batch1["batched_arrivals"] - batch0["batched_arrivals"])) * P
-        b = BYTES_PER_PARAM.get(kind, BYTES_PER_PARAM.get(kind + "_" + wname, 0))
-        return b * P * n
+    def timed_region(max_batch, first_step):
+        """W warm-up + K timed steps starting at window `first_step`; returns the measurements."""
+        def step(s):
+            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
+            h.replay(win, producer_dev, want_log=False, max_batch=max_batch)
+        for s in range(first_step, first_step + args.warmup):
+            step(s)
+        torch.cuda.synchronize(dev)
+        h.timing_enable(True)
+        launches0, batch0 = h.info()["launches"], h.batch_info()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(local_rank) as clk:
+            e0.record()
+            for s in range(first_step + args.warmup, first_step + n_steps):
+                step(s)
+            e1.record()
+            torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        elapsed_ms = e0.elapsed_time(e1)
+        launches = h.info()["launches"] - launches0
+        timing, batch1 = h.timing_read(), h.batch_info()
+        h.timing_enable(False)
+        units = float(args.steps * args.events_per_step) * P
+        t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
+        n_multi = batch1["multi_launches"] - batch0["multi_launches"]
+        n_batched = batch1["batched_arrivals"] - batch0["batched_arrivals"]
 
-    per_kernel = {k: {"launches": n, "mean_ms": (ms / n if n else None), "share_of_step": ms / elapsed_ms,
-                      "GBps": (kernel_bytes(k, n) / 1e9 / (ms * 1e-3) if n else None)} for k, (n, ms) in timing.items()}
-    dominant = max(timing, key=lambda k: timing[k][1])
-    dn, dms = timing[dominant]
-    d_bytes = kernel_bytes(dominant, dn) / dn
-    achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
-    tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
-    roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": (tpp * P if tpp else None), "peak_source": f"of {peak_kind}",
-                "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel,
-                "arrivals_per_multi_launch": ((batch1["batched_arrivals"] - batch0["batched_arrivals"])
-                                              / max(1, batch1["multi_launches"] - batch0["multi_launches"]))}
+        def kernel_bytes(kind, n):
+            """algorithmic bytes of all timed launches of one kernel kind"""
+            if kind == "arrive_multi":
+                return (16 * n_multi + 3 * wbytes * n_batched) * P
+            return BYTES_PER_PARAM.get(kind, BYTES_PER_PARAM.get(kind + "_" + wname, 0)) * P * n
+
+        per_kernel = {k: {"launches": n, "mean_ms": (ms / n if n else None), "share_of_step": ms / elapsed_ms,
+                          "GBps": (kernel_bytes(k, n) / 1e9 / (ms * 1e-3) if n else None)} for k, (n, ms) in timing.items()}
+        dominant = max(timing, key=lambda k: timing[k][1])
+        dn, dms = timing[dominant]
+        d_bytes = kernel_bytes(dominant, dn) / dn
+        achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
+        tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
+        roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": (tpp * P if tpp else None),
+                    "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel}
+        if n_multi:
+            roofline["arrivals_per_multi_launch"] = n_batched / n_multi
+        return {"value": units_all / (t_ms * 1e-3), "ms_per_step": t_ms / args.steps, "launches": int(launches),
+                "roofline": roofline, "clocks": clk.summary()}
+
+    per_event = timed_region(1, 0)                       # one kernel per event
+    if args.max_batch > 1:
+        main_run = timed_region(args.max_batch, n_steps)  # multi-event fusion in the driver
+    else:
+        main_run = per_event
+    value, roofline, launches = main_run["value"], main_run["roofline"], main_run["launches"]
+    t_ms = main_run["ms_per_step"] * args.steps
 
     # ---- end to end (host-resident worker results) ----
     e2e = None
@@ -460,7 +470,7 @@ def main():
         probe = [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]
         from paper_2506_04531_b200.inputs import trace as tr
         e2e_steps = max(1, min(args.steps, 3))
-        base = n_steps
+        base = 2 * n_steps
         run_step(base, e2e=True, host_results=host_results, probe=probe)            # warm-up (allocates staging)
         torch.cuda.synchronize(dev)
         if world > 1:
@@ -495,8 +505,11 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": t_ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "cpu_baseline": cpu}
+                "clocks": main_run["clocks"], "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline, "cpu_baseline": cpu,
+                "per_event_kernels": {"value": per_event["value"], "unit": UNIT, "ms_per_step": per_event["ms_per_step"],
+                                      "gpu_launches": per_event["launches"], "roofline": per_event["roofline"],
+                                      "note": "same workload with one kernel launch per event (max_batch = 1)"}}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -33,6 +33,8 @@ EVENT_DTYPE = np.dtype([("kind", np.uint8), ("lps", np.uint8), ("worker", np.uin
 GBPS_TO_GPS_REGION = (100.0, 0.537, 0.935, 0.202)
 GBPS_INTRA = 100.0
 H_LOCAL_STEPS = 8
+# Relative speeds of the paper's 16 workers, four per region (its worker-speed table).
+PAPER_WORKER_SPEEDS = (10.0, 9.1, 3.8, 2.6, 9.4, 8.0, 6.3, 5.8, 9.9, 5.7, 2.1, 1.5, 9.1, 8.7, 5.8, 1.2)
 
 _M64 = (1 << 64) - 1
 
@@ -69,6 +71,9 @@ class TraceSpec:
     bytes_per_param: int = 4
     lps_gbps: Optional[Sequence[float]] = None   # LPS -> GPS bandwidth; default by region
     h_steps: int = H_LOCAL_STEPS
+    dyn_updates: bool = False        # dynamic local updates: H scaled with worker speed, so that all
+                                     # workers finish a round in the time the fastest needs for H steps
+    bandwidth_scale: float = 1.0     # multiplies every link bandwidth (the paper's 2x-bandwidth study)
 
 
 def generate_trace(spec: TraceSpec) -> np.ndarray:
@@ -78,11 +83,15 @@ def generate_trace(spec: TraceSpec) -> np.ndarray:
     lps_gbps = list(spec.lps_gbps) if spec.lps_gbps is not None else [
         GBPS_TO_GPS_REGION[l % len(GBPS_TO_GPS_REGION)] for l in range(n_lps)]
     model_bytes = spec.P * spec.bytes_per_param
-    hop = transfer_ns(model_bytes, GBPS_INTRA)
+    hop = transfer_ns(model_bytes, GBPS_INTRA * spec.bandwidth_scale)
     s_max = max(spec.speeds)
-    round_ns = [2 * hop + int(round(spec.h_steps * spec.t_profiled_ms * 1e6 * s_max / s))
-                for s in spec.speeds]
-    link_ns = [transfer_ns(model_bytes, g) for g in lps_gbps]
+    if spec.dyn_updates:
+        # H_w = H * S_w / S_max local steps, each taking T_prof * S_max / S_w: every round costs H * T_prof
+        round_ns = [2 * hop + int(round(spec.h_steps * spec.t_profiled_ms * 1e6)) for _ in spec.speeds]
+    else:
+        round_ns = [2 * hop + int(round(spec.h_steps * spec.t_profiled_ms * 1e6 * s_max / s))
+                    for s in spec.speeds]
+    link_ns = [transfer_ns(model_bytes, g * spec.bandwidth_scale) for g in lps_gbps]
 
     heap = [(round_ns[w], ARRIVE, spec.worker_lps[w], w) for w in range(n_workers)]
     heapq.heapify(heap)

@@ -7,13 +7,13 @@ worker speeds, profiled step times of Pythia-70M/160M/410M on one H100: 238.4, 6
 from __future__ import annotations
 
 from dataclasses import dataclass
-from typing import List
+from typing import List, Optional, Sequence
 
 import numpy as np
 
 from . import gen
 from .layouts import Layout, named_layout
-from .trace import TraceSpec, generate_trace, worker_speeds
+from .trace import GBPS_TO_GPS_REGION, PAPER_WORKER_SPEEDS, TraceSpec, generate_trace, worker_speeds
 
 
 @dataclass
@@ -33,14 +33,23 @@ class Workload:
     beta_g: float = 0.5
     alpha: float = 0.25
     slow_region_factor: float = 1.0   # speeds of the last region's workers are divided by this
+    fixed_speeds: Optional[Sequence[float]] = None   # e.g. the paper's 16 worker speeds
+    fixed_worker_lps: Optional[Sequence[int]] = None  # non-uniform grouping of workers under LPSs
+    lps_gbps: Optional[Sequence[float]] = None        # LPS -> GPS link of each LPS (default: by region l % 4)
+    dyn_updates: bool = False
+    bandwidth_scale: float = 1.0
 
     @property
     def worker_lps(self) -> List[int]:
+        if self.fixed_worker_lps is not None:
+            return list(self.fixed_worker_lps)
         per = self.n_workers // self.n_lps
         return [w // per for w in range(self.n_workers)]
 
     @property
     def speeds(self) -> List[float]:
+        if self.fixed_speeds is not None:
+            return list(self.fixed_speeds)
         s = worker_speeds(self.n_workers, self.seed)
         if self.slow_region_factor != 1.0:
             wl = self.worker_lps
@@ -50,7 +59,8 @@ class Workload:
     def trace(self, n_arrivals: int | None = None) -> np.ndarray:
         return generate_trace(TraceSpec(
             P=self.layout.P, worker_lps=self.worker_lps, speeds=self.speeds,
-            t_profiled_ms=self.t_profiled_ms, n_arrivals=n_arrivals or self.n_arrivals, K=self.K))
+            t_profiled_ms=self.t_profiled_ms, n_arrivals=n_arrivals or self.n_arrivals, K=self.K,
+            lps_gbps=self.lps_gbps, dyn_updates=self.dyn_updates, bandwidth_scale=self.bandwidth_scale))
 
     def hyper(self) -> dict:
         return dict(eta_l=self.eta_l, beta_l=self.beta_l, eta_g=self.eta_g, beta_g=self.beta_g,
@@ -58,7 +68,8 @@ class Workload:
 
 
 def workload(name: str) -> Workload:
-    """toy | toy_k4 | 70m | 160m | 410m | 70m_f32_small  (hyperparameters: the paper's selected values)."""
+    """toy | toy_k4 | 70m | 160m | 410m | 70m_f32_small | paper_cluster | paper_cluster_small |
+    hetero_grouping_small  (hyperparameters: the paper's selected values)."""
     if name == "toy":
         return Workload("toy", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1)
     if name == "toy_k4":
@@ -70,6 +81,23 @@ def workload(name: str) -> Workload:
     if name == "410m":
         return Workload("410m", named_layout("410m"), 32, 4, gen.F32, 1589.7, 2000, seed=4,
                         slow_region_factor=3.0)
+    if name == "paper_cluster":
+        # the paper's own simulated cluster: 4 regions x 4 workers with its 16 worker speeds, one LPS
+        # per region, dynamic local updates, 160M layout
+        return Workload("paper_cluster", named_layout("160m"), 16, 4, gen.F32, 623.0, 2000, seed=7,
+                        fixed_speeds=PAPER_WORKER_SPEEDS, dyn_updates=True)
+    if name == "paper_cluster_small":
+        # same cluster structure on a 2^20-parameter vector (cheap enough to check every event)
+        return Workload("paper_cluster_small", named_layout("toy"), 16, 4, gen.F32, 238.4, 400, seed=7, K=8,
+                        fixed_speeds=PAPER_WORKER_SPEEDS, dyn_updates=True)
+    if name == "hetero_grouping_small":
+        # heterogeneous regions with 2, 4, 4, 6 workers under "consistent grouping": 1, 2, 2, 3 LPSs
+        # (two workers each), K = 8, twice the link bandwidth
+        wl_map = [l for l in range(8) for _ in range(2)]
+        region_of_lps = [0, 1, 1, 2, 2, 3, 3, 3]
+        return Workload("hetero_grouping_small", named_layout("toy"), 16, 8, gen.F32, 238.4, 400, seed=8, K=8,
+                        fixed_speeds=PAPER_WORKER_SPEEDS, fixed_worker_lps=wl_map,
+                        lps_gbps=[GBPS_TO_GPS_REGION[r] for r in region_of_lps], bandwidth_scale=2.0)
     if name == "70m_f32_small":
         # profiling case: 70M layout, fp32 copies, 2 workers on 1 LPS (~3 GB on the device, every
         # buffer still larger than L2); K=8 so that pushes, GPS updates and merges occur early

@@ -137,7 +137,7 @@ def test_chunk_size_invariance(chunk):
 # ---------------------------------------------------------------------------------------------
 # configuration 1 ("toy"): 1,048,576 parameters, 4 workers, 2 LPS, 200 arrivals, every event checked
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["toy", "toy_k4"])
+@pytest.mark.parametrize("name", ["toy", "toy_k4", "paper_cluster_small", "hetero_grouping_small"])
 def test_toy_config_every_event(name):
     wl = workloads.workload(name)
     ls = Lockstep(wl.layout, wl.worker_lps, wl.hyper(), wl.worker_dtype, wl.seed)
@@ -145,7 +145,7 @@ def test_toy_config_every_event(name):
     assert ls.bit_identical and ls.max_err <= PER_EVENT_TOL
     # the trace exercised the whole hierarchy
     kinds = [r["kind"] for r in ls.log]
-    assert kinds.count(tr.GPS_RECV) >= (20 if name == "toy_k4" else 4)
+    assert kinds.count(tr.GPS_RECV) >= (4 if name == "toy" else 20)
     assert max(r.get("worker_staleness", 0) for r in ls.log) >= 1
     ls.close()
 

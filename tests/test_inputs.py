@@ -76,7 +76,8 @@ def test_worker_result_dtypes_and_scales():
     np.testing.assert_array_equal(gen.bf16_bits_to_f32(lib), torch.from_numpy(x).to(torch.bfloat16).float().numpy())
 
 
-@pytest.mark.parametrize("name", ["toy", "toy_k4", "70m", "160m", "410m"])
+@pytest.mark.parametrize("name", ["toy", "toy_k4", "70m", "160m", "410m", "paper_cluster", "paper_cluster_small",
+                                  "hetero_grouping_small"])
 def test_trace_structure(name):
     wl = workloads.workload(name)
     ev = wl.trace()
@@ -123,3 +124,33 @@ def test_trace_heterogeneity():
     # a worker's arrivals are evenly spaced by its round time
     w0 = arr[arr["worker"] == 0]["time_ns"]
     assert len(set(np.diff(w0).tolist())) == 1
+
+
+def test_paper_cluster_options():
+    wl = workloads.workload("paper_cluster_small")
+    assert len(wl.speeds) == 16 and max(wl.speeds) == 10.0 and min(wl.speeds) == 1.2
+    ev = wl.trace()
+    arr = ev[ev["kind"] == tr.ARRIVE]
+    # dynamic local updates: every worker needs the same time per round, so arrivals come in
+    # synchronous waves of all 16 workers
+    counts = [int((arr["worker"] == w).sum()) for w in range(16)]
+    assert max(counts) - min(counts) <= 1
+    # without them the fastest worker arrives ~8x as often as the slowest (speeds 10.0 vs 1.2)
+    spec = tr.TraceSpec(P=wl.layout.P, worker_lps=wl.worker_lps, speeds=wl.speeds, t_profiled_ms=238.4,
+                        n_arrivals=400, K=8)
+    arr2 = tr.generate_trace(spec)
+    arr2 = arr2[arr2["kind"] == tr.ARRIVE]
+    c2 = [int((arr2["worker"] == w).sum()) for w in range(16)]
+    assert c2[0] > 6 * c2[15]
+    # doubling the bandwidth shortens every LPS<->GPS round trip
+    g1 = tr.generate_trace(spec)
+    spec2 = tr.TraceSpec(P=wl.layout.P, worker_lps=wl.worker_lps, speeds=wl.speeds, t_profiled_ms=238.4,
+                         n_arrivals=400, K=8, bandwidth_scale=2.0)
+    g2 = tr.generate_trace(spec2)
+    rt = lambda g, l: (g[(g["kind"] == tr.PULL) & (g["lps"] == l)]["time_ns"][0]
+                       - g[(g["kind"] == tr.GPS_RECV) & (g["lps"] == l)]["time_ns"][0])
+    assert rt(g2, 3) * 2 == pytest.approx(rt(g1, 3), rel=1e-6)
+    # consistent grouping: 8 LPSs of two workers each, the last three share region 4's slow link
+    hg = workloads.workload("hetero_grouping_small")
+    assert hg.n_lps == 8 and sorted(set(hg.worker_lps)) == list(range(8))
+    assert hg.lps_gbps[5] == hg.lps_gbps[7] == 0.202 and hg.lps_gbps[0] == 100.0
