@@ -27,7 +27,8 @@ _SOURCES = [_HERE / "halos_oracle_c.cpp", _HERE / "halos_oracle.hpp"]
 
 F32, BF16 = 0, 1
 IDLE, PUSHED, ANSWERED = 0, 1, 2
-_WHICH = {"Theta": 0, "Mg": 1, "th": 2, "ml": 3, "anchor": 4, "outbox": 5, "inbox": 6, "th0": 7, "delta": 8}
+OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1
+_WHICH = {"Theta": 0, "Mg": 1, "th": 2, "ml": 3, "anchor": 4, "outbox": 5, "inbox": 6, "th0": 7, "delta": 8, "acc": 9, "acc_g": 10}
 
 
 def build(force: bool = False) -> Path:
@@ -56,7 +57,7 @@ def _load():
     lib.halos_oracle_create.restype = c.c_void_p
     lib.halos_oracle_create.argtypes = [c.c_int, c.c_uint64, c.c_uint32, c.c_uint32, c.c_void_p,
                                         c.c_double, c.c_double, c.c_double, c.c_double, c.c_double,
-                                        c.c_uint32, c.c_int, c.c_void_p]
+                                        c.c_uint32, c.c_int, c.c_void_p, c.c_int, c.c_uint32, c.c_uint32]
     lib.halos_oracle_destroy.argtypes = [c.c_void_p]
     lib.halos_oracle_error.restype = c.c_char_p
     lib.halos_oracle_error.argtypes = [c.c_void_p]
@@ -93,11 +94,13 @@ class HalosOracle:
     ``dtype`` is the scalar type of the master state: ``np.float32`` (parity oracle) or
     ``np.float64`` (self-check oracle).  ``worker_dtype`` is F32 or BF16: the type worker
     snapshots theta_{t,0} are stored in and worker results theta_{t,H} are given in
-    (bf16 as uint16 bit patterns).
+    (bf16 as uint16 bit patterns).  ``optimizer=OPT_DELAYED_NESTEROV`` with ``delay_l/delay_g`` selects the
+    delayed-Nesterov reading described in halos_oracle.hpp (then eta_l/eta_g are its unscaled rates).
     """
 
     def __init__(self, theta_init, worker_lps, *, n_lps=None, eta_l=0.2, beta_l=0.9, eta_g=0.15,
-                 beta_g=0.5, alpha=0.25, K=32, worker_dtype=F32, dtype=np.float32):
+                 beta_g=0.5, alpha=0.25, K=32, worker_dtype=F32, dtype=np.float32,
+                 optimizer=OPT_PAPER, delay_l=1, delay_g=1):
         lib = _load()
         theta_init = np.ascontiguousarray(theta_init, dtype=np.float32)
         wl = np.ascontiguousarray(worker_lps, dtype=np.uint32)
@@ -113,7 +116,8 @@ class HalosOracle:
         self._h = lib.halos_oracle_create(int(self.dtype == np.float64), self.P, self.n_lps,
                                           self.n_workers, wl.ctypes.data, float(eta_l), float(beta_l),
                                           float(eta_g), float(beta_g), float(alpha), int(K),
-                                          self.worker_dtype, theta_init.ctypes.data)
+                                          self.worker_dtype, theta_init.ctypes.data, int(optimizer),
+                                          int(delay_l), int(delay_g))
         if not self._h:
             raise OracleError("halos_oracle_create failed")
 

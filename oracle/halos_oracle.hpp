@@ -30,6 +30,18 @@
 //   * Delta is not divided by K.
 //   * Rounding order: each fma below is one fused multiply-add (single rounding); every
 //     other product or difference is rounded on its own.  Compile with -ffp-contract=off.
+//
+// Optional optimizer OPT_DELAYED_NESTEROV.  The paper's experiments replace ModelUpdate by the
+// "delayed Nesterov" optimizer of the Async-Local-SGD work it cites, but never define it; the only
+// property it states is that the rule "effectively divides the learning rate by the delay interval"
+// (hyperparameter table, Appendix D).  The reading implemented here, per server with delay d,
+// rate eps, an accumulator acc and n = number of updates seen so far:
+//     acc += g                                        every update
+//     n mod d != 0:  theta -= (eps/d) g               momentum untouched
+//     n mod d == 0:  m = beta m + acc/d ;  theta -= eps (beta m + g/d) ;  acc = 0
+// (g = -displacement as above).  THE READING IS UNPINNED BY THE PAPER; the implementation is
+// pinned to the stated property (mean step eps g / (d (1-beta)) under constant g), to textbook
+// Nesterov SGD for d = 1, and to an independent interpreter.
 #pragma once
 #include <cmath>
 #include <cstdint>
@@ -41,6 +53,7 @@ namespace halos_oracle {
 
 enum WorkerDtype { W_F32 = 0, W_BF16 = 1 };
 enum Phase { IDLE = 0, PUSHED = 1, ANSWERED = 2 };
+enum Optimizer { OPT_PAPER = 0, OPT_DELAYED_NESTEROV = 1 };
 
 // fp32 -> bf16, round to nearest, ties to even; result is the upper 16 bits.
 // Written out on integers so that it does not depend on any hardware conversion.
@@ -69,12 +82,15 @@ struct Config {
     double alpha = 0.25;               // merging weight
     uint32_t K = 32;                   // local updates accumulated per push
     int worker_dtype = W_F32;
+    int optimizer = OPT_PAPER;
+    uint32_t delay_l = 1, delay_g = 1;  // momentum refresh interval of the LPSs / the GPS (delayed Nesterov only)
 };
 
 template <class T>
 struct Lps {
     std::vector<T> th, ml, anchor, outbox, inbox;
     std::vector<T> last_delta;  // the worker displacement applied by the most recent arrival (observability)
+    std::vector<T> acc;         // delayed Nesterov: displacements accumulated since the last momentum refresh
     uint64_t t = 0, t_last = 0, t_push = 0;
     int phase = IDLE;
 };
@@ -84,6 +100,7 @@ class Oracle {
 public:
     Config cfg;
     std::vector<T> Theta, Mg;
+    std::vector<T> acc_g;  // delayed Nesterov accumulator of the GPS
     uint64_t i = 0;
     std::vector<Lps<T>> lps;
     std::vector<std::vector<float>> th0_f32;      // worker snapshots when worker_dtype == W_F32
@@ -100,6 +117,8 @@ public:
         const uint64_t P = c.P;
         Theta.resize(P);
         Mg.assign(P, T(0));
+        acc_g.assign(P, T(0));
+        if (c.delay_l == 0 || c.delay_g == 0) throw std::invalid_argument("delay must be >= 1");
         for (uint64_t j = 0; j < P; ++j) Theta[j] = (T)theta_init[j];
         lps.resize(c.n_lps);
         for (auto& s : lps) {
@@ -109,6 +128,7 @@ public:
             s.outbox.assign(P, T(0));
             s.inbox.assign(P, T(0));
             s.last_delta.assign(P, T(0));
+            s.acc.assign(P, T(0));
         }
         worker_round.assign(c.n_workers, 0);
         worker_sched_t.assign(c.n_workers, 0);
@@ -132,6 +152,27 @@ public:
         m = m_new;
     }
 
+    // Delayed Nesterov step on one element with displacement d (see the header for the reading).
+    static inline void delayed_nesterov(T& theta, T& m, T& acc, T d, T eps, T beta, T inv_delay, T eps_over_delay,
+                                        bool refresh) {
+        acc = acc + d;
+        if (!refresh) {
+            theta = std::fma(eps_over_delay, d, theta);        // theta' = theta + (eps/d) d
+        } else {
+            T m_new = std::fma(beta, m, acc * inv_delay);      // m' = beta m + acc/d
+            T u = std::fma(beta, m_new, d * inv_delay);        // beta m' + d/d
+            theta = std::fma(eps, u, theta);
+            m = m_new;
+            acc = T(0);
+        }
+    }
+
+    // One server-side optimizer step of the configured kind on element (theta, m, acc).
+    inline void step(T& theta, T& m, T& acc, T d, T eta, T beta, T omb, T inv_delay, T eta_over_delay, bool refresh) const {
+        if (cfg.optimizer == OPT_PAPER) model_update(theta, m, d, eta, beta, omb);
+        else delayed_nesterov(theta, m, acc, d, eta, beta, inv_delay, eta_over_delay, refresh);
+    }
+
     // A worker's result theta_{t,H} reaches its LPS (Alg. 1 lines 9-15 and 25).
     // thetaH is in the worker dtype (float, or uint16_t bf16 patterns).  Returns true if the
     // arrival completed a window of K updates, in which case Delta was formed (line 14).
@@ -139,6 +180,8 @@ public:
         if (w >= cfg.n_workers) throw std::invalid_argument("worker out of range");
         Lps<T>& s = lps[cfg.worker_lps[w]];
         const T eta = (T)cfg.eta_l, beta = (T)cfg.beta_l, omb = T(1) - beta;
+        const T inv_delay = T(1) / (T)cfg.delay_l, eta_over_delay = eta * inv_delay;
+        const bool refresh = ((s.t + 1) % cfg.delay_l) == 0;   // this is the LPS's update number t+1
         const uint64_t P = cfg.P;
         if (cfg.worker_dtype == W_F32) {
             const float* h = (const float*)thetaH;
@@ -146,7 +189,7 @@ public:
             for (uint64_t j = 0; j < P; ++j) {
                 T d = (T)h[j] - (T)s0[j];                  // line 25: delta = theta_{t,H} - theta_{t,0}
                 s.last_delta[j] = d;
-                model_update(s.th[j], s.ml[j], d, eta, beta, omb);   // line 11
+                step(s.th[j], s.ml[j], s.acc[j], d, eta, beta, omb, inv_delay, eta_over_delay, refresh);   // line 11
                 s0[j] = (float)s.th[j];                    // line 12: schedule the worker theta_t
             }
         } else {
@@ -155,7 +198,7 @@ public:
             for (uint64_t j = 0; j < P; ++j) {
                 T d = (T)bf16_to_f32(h[j]) - (T)bf16_to_f32(s0[j]);
                 s.last_delta[j] = d;
-                model_update(s.th[j], s.ml[j], d, eta, beta, omb);
+                step(s.th[j], s.ml[j], s.acc[j], d, eta, beta, omb, inv_delay, eta_over_delay, refresh);
                 s0[j] = f32_to_bf16_rne((float)s.th[j]);
             }
         }
@@ -184,8 +227,10 @@ public:
         Lps<T>& s = lps.at(l);
         if (s.phase != PUSHED) throw std::logic_error("gps_recv without a pushed Delta");
         const T eta = (T)cfg.eta_g, beta = (T)cfg.beta_g, omb = T(1) - beta;
+        const T inv_delay = T(1) / (T)cfg.delay_g, eta_over_delay = eta * inv_delay;
+        const bool refresh = ((i + 1) % cfg.delay_g) == 0;
         for (uint64_t j = 0; j < cfg.P; ++j) {
-            model_update(Theta[j], Mg[j], s.outbox[j], eta, beta, omb);
+            step(Theta[j], Mg[j], acc_g[j], s.outbox[j], eta, beta, omb, inv_delay, eta_over_delay, refresh);
             s.inbox[j] = Theta[j];
         }
         i += 1;

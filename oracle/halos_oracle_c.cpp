@@ -30,13 +30,13 @@ int guarded(Handle* h, F&& fn) {
 
 extern "C" {
 
-// which: 0 Theta, 1 Mg, 2 th[l], 3 ml[l], 4 anchor[l], 5 outbox[l], 6 inbox[l], 7 th0[w], 8 last delta[l]
-enum { B_THETA = 0, B_MG, B_TH, B_ML, B_ANCHOR, B_OUTBOX, B_INBOX, B_TH0, B_DELTA };
+// which: 0 Theta, 1 Mg, 2 th[l], 3 ml[l], 4 anchor[l], 5 outbox[l], 6 inbox[l], 7 th0[w], 8 last delta[l], 9 acc[l], 10 acc_g
+enum { B_THETA = 0, B_MG, B_TH, B_ML, B_ANCHOR, B_OUTBOX, B_INBOX, B_TH0, B_DELTA, B_ACC_L, B_ACC_G };
 
 void* halos_oracle_create(int use_double, uint64_t P, uint32_t n_lps, uint32_t n_workers,
                           const uint32_t* worker_lps, double eta_l, double beta_l, double eta_g,
                           double beta_g, double alpha, uint32_t K, int worker_dtype,
-                          const float* theta_init) {
+                          const float* theta_init, int optimizer, uint32_t delay_l, uint32_t delay_g) {
     Config c;
     c.P = P;
     c.n_lps = n_lps;
@@ -49,6 +49,9 @@ void* halos_oracle_create(int use_double, uint64_t P, uint32_t n_lps, uint32_t n
     c.alpha = alpha;
     c.K = K;
     c.worker_dtype = worker_dtype;
+    c.optimizer = optimizer;
+    c.delay_l = delay_l;
+    c.delay_g = delay_g;
     Handle* h = new Handle();
     h->is_double = use_double;
     h->f = nullptr;
@@ -107,6 +110,8 @@ void* halos_oracle_buffer(void* hv, int which, uint32_t idx) {
             case B_ANCHOR: return idx < o->lps.size() ? o->lps[idx].anchor.data() : nullptr;
             case B_OUTBOX: return idx < o->lps.size() ? o->lps[idx].outbox.data() : nullptr;
             case B_INBOX: return idx < o->lps.size() ? o->lps[idx].inbox.data() : nullptr;
+            case B_ACC_L: return idx < o->lps.size() ? o->lps[idx].acc.data() : nullptr;
+            case B_ACC_G: return o->acc_g.data();
             case B_DELTA: return idx < o->lps.size() ? o->lps[idx].last_delta.data() : nullptr;
             case B_TH0:
                 if (idx >= o->cfg.n_workers) return nullptr;
