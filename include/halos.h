@@ -47,6 +47,18 @@ enum {
 
 enum { HALOS_F32 = 0, HALOS_BF16 = 1 };
 
+/* Server-side optimizer.
+ * HALOS_OPT_PAPER: the ModelUpdate rule the paper defines (Appendix E); the default.
+ * HALOS_OPT_DELAYED_NESTEROV: the optimizer the paper's experiments used ("delayed Nesterov", cited from
+ * the Async-Local-SGD work, never defined in the paper; its hyperparameter table only says that the
+ * rule "effectively divides the learning rate by the delay interval").  Reading implemented, per server
+ * with delay n, rate eps (= eta_l / eta_g), accumulator acc, k = number of updates seen so far:
+ *     acc += d                                            every update (d = displacement)
+ *     k mod n != 0:   x += (eps/n) d                      momentum untouched
+ *     k mod n == 0:   m = beta m + acc/n ;  x += eps (beta m + d/n) ;  acc = 0
+ * The paper's selected values in this mode: delay_l = 16, eta_l = 3.2, delay_g = 2, eta_g = 0.3. */
+enum { HALOS_OPT_PAPER = 0, HALOS_OPT_DELAYED_NESTEROV = 1 };
+
 /* flags */
 enum {
     HALOS_FLAG_STATS = 1u          /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
@@ -64,7 +76,9 @@ enum {
     HALOS_BUF_ANCHOR = 4,   /* theta_{t_last} of LPS index */
     HALOS_BUF_OUTBOX = 5,   /* Delta in flight from LPS index */
     HALOS_BUF_INBOX = 6,    /* Theta_i in flight to LPS index */
-    HALOS_BUF_THETA0 = 7    /* start snapshot of worker index (worker_dtype) */
+    HALOS_BUF_THETA0 = 7,   /* start snapshot of worker index (worker_dtype) */
+    HALOS_BUF_ACC_L = 8,    /* delayed Nesterov accumulator of LPS index  (that optimizer only) */
+    HALOS_BUF_ACC_G = 9     /* delayed Nesterov accumulator of the GPS    (that optimizer only) */
 };
 
 typedef struct halos_config {
@@ -88,6 +102,8 @@ typedef struct halos_config {
     void (*free_)(void* ptr, void* user);
     void* alloc_user;
     uint32_t chunk_elems;          /* scheduler chunk size in elements; 0 = library default */
+    uint32_t optimizer;            /* HALOS_OPT_PAPER | HALOS_OPT_DELAYED_NESTEROV */
+    uint32_t delay_l, delay_g;     /* momentum refresh interval of the LPSs / the GPS (delayed Nesterov; >= 1) */
     uint32_t reserved;
 } halos_config;
 

@@ -22,7 +22,8 @@ OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED = range(6
 F32, BF16 = 0, 1
 FLAG_STATS = 1
 IDLE, PUSHED, ANSWERED = 0, 1, 2
-BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0 = range(8)
+BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0, BUF_ACC_L, BUF_ACC_G = range(10)
+OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1
 EV_ARRIVE, EV_GPS_RECV, EV_PULL = 0, 1, 2
 K_ARRIVE, K_ARRIVE_PUSH, K_PUSH, K_GPS, K_PULL, K_ARRIVE_MULTI = range(6)
 KERNEL_NAMES = ("arrive", "arrive_push", "push", "gps", "pull", "arrive_multi")
@@ -51,7 +52,8 @@ class Config(C.Structure):
         ("alpha", C.c_float), ("K", C.c_uint32), ("worker_dtype", C.c_uint32), ("flags", C.c_uint32),
         ("device", C.c_int32), ("stream", C.c_void_p),
         ("alloc", ALLOC_FN), ("free_", FREE_FN), ("alloc_user", C.c_void_p),
-        ("chunk_elems", C.c_uint32), ("reserved", C.c_uint32),
+        ("chunk_elems", C.c_uint32), ("optimizer", C.c_uint32), ("delay_l", C.c_uint32), ("delay_g", C.c_uint32),
+        ("reserved", C.c_uint32),
     ]
 
 
@@ -161,7 +163,7 @@ class Halos:
     def __init__(self, theta_init, worker_lps: Sequence[int], tensor_numel: Optional[Sequence[int]] = None, *,
                  n_lps: Optional[int] = None, eta_l=0.2, beta_l=0.9, eta_g=0.15, beta_g=0.5, alpha=0.25, K=32,
                  worker_dtype=F32, flags=0, chunk_elems=0, stream=None, use_torch_allocator=True,
-                 alloc_limit_bytes: Optional[int] = None):
+                 alloc_limit_bytes: Optional[int] = None, optimizer=OPT_PAPER, delay_l=1, delay_g=1):
         import torch
         self._torch = torch
         if not torch.cuda.is_available():
@@ -210,6 +212,7 @@ class Halos:
         cfg.tensor_numel = tn.ctypes.data_as(C.POINTER(C.c_uint64))
         cfg.eta_l, cfg.beta_l, cfg.eta_g, cfg.beta_g, cfg.alpha = eta_l, beta_l, eta_g, beta_g, alpha
         cfg.K, cfg.worker_dtype, cfg.flags, cfg.chunk_elems = int(K), self.worker_dtype, int(flags), int(chunk_elems)
+        cfg.optimizer, cfg.delay_l, cfg.delay_g = int(optimizer), int(delay_l), int(delay_g)
         cfg.device = self.device.index if self.device.index is not None else torch.cuda.current_device()
         cfg.stream = self._stream.cuda_stream
         if use_torch_allocator:

@@ -24,6 +24,7 @@ thread_local std::string g_create_error;
 
 struct LpsState {
     float *th = nullptr, *ml = nullptr, *anchor = nullptr, *outbox = nullptr, *inbox = nullptr;
+    float* acc = nullptr;  // delayed Nesterov only
     uint64_t t = 0, t_last = 0, t_push = 0;
     uint64_t inbox_iter = 0;  // GPS iteration that produced the inbox content
     int phase = HALOS_IDLE;
@@ -69,6 +70,7 @@ struct halos_ctx {
     double* d_stats = nullptr;  // [2][n_lps][n_tensors]
 
     float *Theta = nullptr, *Mg = nullptr;
+    float* acc_g = nullptr;  // delayed Nesterov only
     uint64_t gps_iter = 0;
     std::vector<LpsState> lps;
     std::vector<WorkerState> workers;
@@ -198,7 +200,41 @@ struct Timer {
 };
 
 template <class W>
+int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
+    ArriveDnArgs<W> a;
+    a.h_flat = (const W*)flat;
+    a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)widx * c->tensor_numel.size());
+    a.tensor_off = c->d_tensor_off;
+    a.th0 = (W*)w.th0;
+    a.th = s.th;
+    a.ml = s.ml;
+    a.acc = s.acc;
+    a.anchor = s.anchor;
+    a.outbox = s.outbox;
+    a.eps = c->cfg.eta_l;
+    a.beta = c->cfg.beta_l;
+    a.inv_n = 1.0f / (float)c->cfg.delay_l;
+    a.eps_n = c->cfg.eta_l * a.inv_n;
+    const bool refresh = ((s.t + 1) % c->cfg.delay_l) == 0;   // s.t is advanced after the launch
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    if (grid.x == 0) return HALOS_OK;
+    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+    if (refresh) {
+        if (push) arrive_dn_kernel<W, true, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_dn_kernel<W, true, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    } else {
+        if (push) arrive_dn_kernel<W, false, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_dn_kernel<W, false, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    }
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+
+template <class W>
 int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
+    if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat);
     ArriveArgs<W> a;
     a.h_flat = (const W*)flat;
     a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)widx * c->tensor_numel.size());
@@ -372,6 +408,9 @@ void halos_default_config(halos_config* cfg) {
     cfg->alpha = 0.25f;
     cfg->K = 32;
     cfg->worker_dtype = HALOS_F32;
+    cfg->optimizer = HALOS_OPT_PAPER;
+    cfg->delay_l = 1;
+    cfg->delay_g = 1;
 }
 
 int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx** out) {
@@ -383,6 +422,12 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     if (cfg->K == 0) return fail(nullptr, HALOS_ERR_INVALID_ARG, "K must be positive");
     if (cfg->worker_dtype != HALOS_F32 && cfg->worker_dtype != HALOS_BF16)
         return fail(nullptr, HALOS_ERR_INVALID_ARG, "unknown worker_dtype");
+    if (cfg->optimizer != HALOS_OPT_PAPER && cfg->optimizer != HALOS_OPT_DELAYED_NESTEROV)
+        return fail(nullptr, HALOS_ERR_INVALID_ARG, "unknown optimizer");
+    if (cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV && (cfg->delay_l == 0 || cfg->delay_g == 0))
+        return fail(nullptr, HALOS_ERR_INVALID_ARG, "delays must be at least 1");
+    if (cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV && (cfg->flags & HALOS_FLAG_STATS))
+        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "statistics are not available with the delayed Nesterov optimizer");
     if ((cfg->alloc == nullptr) != (cfg->free_ == nullptr)) return fail(nullptr, HALOS_ERR_INVALID_ARG, "alloc and free_ go together");
     for (uint32_t w = 0; w < cfg->n_workers; ++w)
         if (cfg->worker_lps[w] >= cfg->n_lps) return fail(nullptr, HALOS_ERR_INVALID_ARG, "worker_lps[%u] out of range", w);
@@ -445,6 +490,8 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     }
     ok &= (c->Theta = (float*)A(P * 4)) != nullptr;
     ok &= (c->Mg = (float*)A(P * 4)) != nullptr;
+    const bool dn = cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV;
+    if (dn) ok &= (c->acc_g = (float*)A(P * 4)) != nullptr;
     c->lps.resize(cfg->n_lps);
     for (auto& s : c->lps) {
         if (!ok) break;
@@ -453,6 +500,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
         ok &= (s.anchor = (float*)A(P * 4)) != nullptr;
         ok &= (s.outbox = (float*)A(P * 4)) != nullptr;
         ok &= (s.inbox = (float*)A(P * 4)) != nullptr;
+        if (dn) ok &= (s.acc = (float*)A(P * 4)) != nullptr;
     }
     c->workers.resize(cfg->n_workers);
     for (uint32_t w = 0; w < cfg->n_workers && ok; ++w) {
@@ -479,12 +527,14 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     // Alg. 1 lines 6-7
     CUC(cudaMemcpyAsync(c->Theta, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
     CUC(cudaMemsetAsync(c->Mg, 0, P * 4, st));
+    if (c->acc_g) CUC(cudaMemsetAsync(c->acc_g, 0, P * 4, st));
     for (auto& s : c->lps) {
         CUC(cudaMemcpyAsync(s.th, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
         CUC(cudaMemcpyAsync(s.anchor, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
         CUC(cudaMemsetAsync(s.ml, 0, P * 4, st));
         CUC(cudaMemsetAsync(s.outbox, 0, P * 4, st));
         CUC(cudaMemsetAsync(s.inbox, 0, P * 4, st));
+        if (s.acc) CUC(cudaMemsetAsync(s.acc, 0, P * 4, st));
     }
     for (auto& w : c->workers) {
         if (c->wb == 4) {
@@ -601,10 +651,17 @@ int halos_gps_merge(halos_ctx* c, uint32_t lps) {
     LpsState& s = c->lps[lps];
     if (s.phase != HALOS_PUSHED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Delta in flight", lps);
     CU(c, cudaSetDevice(c->cfg.device));
-    GpsArgs a{s.outbox, c->Theta, c->Mg, s.inbox, c->cfg.eta_g, c->cfg.beta_g, 1.0f - c->cfg.beta_g};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     Timer tm(c, HALOS_K_GPS);
-    gps_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) {
+        const float inv_n = 1.0f / (float)c->cfg.delay_g;
+        GpsDnArgs a{s.outbox, c->Theta, c->Mg, c->acc_g, s.inbox, c->cfg.eta_g, c->cfg.beta_g, inv_n, c->cfg.eta_g * inv_n};
+        if (((c->gps_iter + 1) % c->cfg.delay_g) == 0) gps_dn_kernel<true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else gps_dn_kernel<false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    } else {
+        GpsArgs a{s.outbox, c->Theta, c->Mg, s.inbox, c->cfg.eta_g, c->cfg.beta_g, 1.0f - c->cfg.beta_g};
+        gps_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    }
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
@@ -648,6 +705,7 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
     if (max_batch == 0) max_batch = 1;
     if (max_batch > (uint32_t)kMaxBatch) max_batch = kMaxBatch;
     if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
+    const bool immediate = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV;  // that optimizer is launched event by event
     std::vector<std::vector<Deferred>> queue(c->cfg.n_lps);
     int rc = HALOS_OK;
     uint32_t k = 0;
@@ -680,10 +738,10 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
                 }
                 bool due = false, push = false;
                 if (rc == HALOS_OK) rc = apply_check(c, e.lps, e.worker, true, &due, &push);
-                if (rc == HALOS_OK && w.pending == PEND_STAGED && !q.empty()) rc = flush_deferred(c, e.lps, q, false);
+                if (rc == HALOS_OK && (w.pending == PEND_STAGED || immediate) && !q.empty()) rc = flush_deferred(c, e.lps, q, false);
                 if (rc == HALOS_OK) {
                     rec.worker_staleness = c->lps[e.lps].t - w.sched_t;
-                    if (w.pending == PEND_STAGED) {
+                    if (w.pending == PEND_STAGED || immediate) {
                         rc = apply_impl(c, e.lps, e.worker, true, nullptr);   // host-staged results are not deferred
                     } else {
                         q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr});
@@ -734,7 +792,7 @@ struct CkptHeader {
     uint64_t P;
     uint32_t n_lps, n_workers, n_tensors, K;
     float eta_l, beta_l, eta_g, beta_g, alpha;
-    uint32_t pad;
+    uint32_t optimizer;
     uint64_t gps_iter;
 };
 struct CkptLps { uint64_t t, t_last, t_push, inbox_iter; int32_t phase; int32_t pad; };
@@ -782,6 +840,7 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
         h.n_lps = c->cfg.n_lps; h.n_workers = c->cfg.n_workers; h.n_tensors = c->cfg.n_tensors; h.K = c->cfg.K;
         h.eta_l = c->cfg.eta_l; h.beta_l = c->cfg.beta_l; h.eta_g = c->cfg.eta_g; h.beta_g = c->cfg.beta_g; h.alpha = c->cfg.alpha;
         h.gps_iter = c->gps_iter;
+        h.optimizer = c->cfg.optimizer;
         for (size_t l = 0; l < ls.size(); ++l)
             ls[l] = CkptLps{c->lps[l].t, c->lps[l].t_last, c->lps[l].t_push, c->lps[l].inbox_iter, c->lps[l].phase, 0};
         for (size_t w = 0; w < ws.size(); ++w) ws[w] = CkptWorker{c->workers[w].round, c->workers[w].sched_t};
@@ -792,7 +851,8 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
         std::vector<uint64_t> numel(c->tensor_numel.size());
         if (fread(&h, sizeof h, 1, f) != 1 || std::memcmp(h.magic, "HALOSCK1", 8) != 0 || h.version != 1)
             rc = fail(c, HALOS_ERR_INVALID_ARG, "not a checkpoint file of this library");
-        else if (h.P != c->P || h.wb != c->wb || h.n_lps != c->cfg.n_lps || h.n_workers != c->cfg.n_workers || h.n_tensors != c->cfg.n_tensors)
+        else if (h.P != c->P || h.wb != c->wb || h.n_lps != c->cfg.n_lps || h.n_workers != c->cfg.n_workers || h.n_tensors != c->cfg.n_tensors ||
+                 h.optimizer != c->cfg.optimizer)
             rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint shape does not match this context");
         else if (fread(numel.data(), 8, numel.size(), f) != numel.size() || numel != c->tensor_numel)
             rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint tensor sizes do not match this context");
@@ -804,8 +864,10 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
     };
     pass(c->Theta, c->P * 4);
     pass(c->Mg, c->P * 4);
+    if (c->acc_g) pass(c->acc_g, c->P * 4);
     for (auto& s : c->lps) {
         pass(s.th, c->P * 4); pass(s.ml, c->P * 4); pass(s.anchor, c->P * 4); pass(s.outbox, c->P * 4); pass(s.inbox, c->P * 4);
+        if (s.acc) pass(s.acc, c->P * 4);
     }
     for (auto& w : c->workers) pass(w.th0, c->P * c->wb);
     if (rc == HALOS_OK && !to_file) {
@@ -838,6 +900,14 @@ static int buffer_of(halos_ctx* c, uint32_t which, uint32_t index, const void** 
                  : which == HALOS_BUF_OUTBOX ? s.outbox : s.inbox;
             return HALOS_OK;
         }
+        case HALOS_BUF_ACC_L:
+            if (index >= c->cfg.n_lps || !c->lps[index].acc) return fail(c, HALOS_ERR_INVALID_ARG, "no accumulator (optimizer or lps)");
+            *p = c->lps[index].acc;
+            return HALOS_OK;
+        case HALOS_BUF_ACC_G:
+            if (!c->acc_g) return fail(c, HALOS_ERR_INVALID_ARG, "no accumulator with this optimizer");
+            *p = c->acc_g;
+            return HALOS_OK;
         case HALOS_BUF_THETA0:
             if (index >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "worker out of range");
             *p = c->workers[index].th0;

@@ -55,6 +55,23 @@ __device__ __forceinline__ void model_update(float& x, float& m, float d, float 
     x = __fmaf_rn(eta, u, x);
     m = m1;
 }
+// Delayed-Nesterov step (optional optimizer; the reading is described in include/halos.h):
+//   acc' = acc + d;  plain update: x' = x + (eps/n) d;  refresh: m' = beta m + acc'/n,
+//   x' = x + eps (beta m' + d/n), acc' = 0.   inv_n = 1/n and eps_n = eps * inv_n are fp32 constants.
+template <bool REFRESH>
+__device__ __forceinline__ void delayed_nesterov(float& x, float& m, float& acc, float d, float eps, float beta,
+                                                 float inv_n, float eps_n) {
+    acc = __fadd_rn(acc, d);
+    if (!REFRESH) {
+        x = __fmaf_rn(eps_n, d, x);
+    } else {
+        float m1 = __fmaf_rn(beta, m, __fmul_rn(acc, inv_n));
+        float u = __fmaf_rn(beta, m1, __fmul_rn(d, inv_n));
+        x = __fmaf_rn(eps, u, x);
+        m = m1;
+        acc = 0.f;
+    }
+}
 __device__ __forceinline__ float merge(float x, float y, float alpha, float oma) {
     return __fmaf_rn(alpha, y, __fmul_rn(oma, x));
 }
@@ -407,6 +424,135 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
         th[i] = x;
         ml[i] = m;
         if (PUSH) ob[i] = __fsub_rn(x, an[i]);
+    }
+}
+
+// =====================================================================================================
+// Delayed-Nesterov variants of ARRIVE and GPS.  A plain update touches theta and the accumulator
+// (momentum is neither read nor written: same 16 + 3 w_b bytes per parameter as the paper's rule);
+// a refresh update also reads and writes the momentum (+8 bytes).
+// =====================================================================================================
+template <class W>
+struct ArriveDnArgs {
+    const W* h_flat;
+    const W* const* h_ptrs;
+    const unsigned long long* tensor_off;
+    W* th0;
+    float* th;
+    float* ml;
+    float* acc;
+    const float* anchor;
+    float* outbox;
+    float eps, beta, inv_n, eps_n;
+};
+
+template <class W, bool REFRESH, bool PUSH, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+arrive_dn_kernel(const Chunk* __restrict__ chunks, ArriveDnArgs<W> a) {
+    using T = WTraits<W>;
+    const Chunk c = chunks[blockIdx.x];
+    const W* h = a.h_flat ? a.h_flat + c.begin : a.h_ptrs[c.tensor] + (c.begin - a.tensor_off[c.tensor]);
+    W* s0 = a.th0 + c.begin;
+    float* th = a.th + c.begin;
+    float* ml = a.ml + c.begin;
+    float* ac = a.acc + c.begin;
+    const float* an = PUSH ? a.anchor + c.begin : nullptr;
+    float* ob = PUSH ? a.outbox + c.begin : nullptr;
+    const float eps = a.eps, beta = a.beta, inv_n = a.inv_n, eps_n = a.eps_n;
+    const bool vec_ok = ((c.begin % VE) == 0) && ((reinterpret_cast<uintptr_t>(h) % (VE * sizeof(W))) == 0);
+    uint32_t done = 0;
+    if (vec_ok) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vh = T::template load<VE, STREAM>(h + o);
+            FVec<VE> vs = T::template load<VE, STREAM>(s0 + o);
+            FVec<VE> vx = ldf<VE, STREAM>(th + o);
+            FVec<VE> vc = ldf<VE, STREAM>(ac + o);
+            FVec<VE> vm, va;
+            if (REFRESH) vm = ldf<VE, STREAM>(ml + o);
+            if (PUSH) va = ldf<VE, STREAM>(an + o);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) {
+                const float d = __fsub_rn(vh.v[e], vs.v[e]);
+                float m = REFRESH ? vm.v[e] : 0.f;
+                delayed_nesterov<REFRESH>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
+                if (REFRESH) vm.v[e] = m;
+            }
+            stf<VE, STREAM>(th + o, vx);
+            stf<VE, STREAM>(ac + o, vc);
+            if (REFRESH) stf<VE, STREAM>(ml + o, vm);
+            T::template store<VE, STREAM>(s0 + o, vx);
+            if (PUSH) {
+                FVec<VE> D;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                stf<VE, STREAM>(ob + o, D);
+            }
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
+        const float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
+        float x = th[j], acc = ac[j], m = REFRESH ? ml[j] : 0.f;
+        delayed_nesterov<REFRESH>(x, m, acc, d, eps, beta, inv_n, eps_n);
+        th[j] = x;
+        ac[j] = acc;
+        if (REFRESH) ml[j] = m;
+        T::store1(s0 + j, x);
+        if (PUSH) ob[j] = __fsub_rn(x, an[j]);
+    }
+}
+
+struct GpsDnArgs {
+    const float* outbox;
+    float* Theta;
+    float* Mg;
+    float* acc;
+    float* inbox;
+    float eps, beta, inv_n, eps_n;
+};
+
+template <bool REFRESH, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+gps_dn_kernel(const Chunk* __restrict__ chunks, GpsDnArgs a) {
+    const Chunk c = chunks[blockIdx.x];
+    const float* ob = a.outbox + c.begin;
+    float* Th = a.Theta + c.begin;
+    float* Mg = a.Mg + c.begin;
+    float* ac = a.acc + c.begin;
+    float* ib = a.inbox + c.begin;
+    const float eps = a.eps, beta = a.beta, inv_n = a.inv_n, eps_n = a.eps_n;
+    uint32_t done = 0;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vd = ldf<VE, STREAM>(ob + o);
+            FVec<VE> vx = ldf<VE, STREAM>(Th + o);
+            FVec<VE> vc = ldf<VE, STREAM>(ac + o);
+            FVec<VE> vm;
+            if (REFRESH) vm = ldf<VE, STREAM>(Mg + o);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) {
+                float m = REFRESH ? vm.v[e] : 0.f;
+                delayed_nesterov<REFRESH>(vx.v[e], m, vc.v[e], vd.v[e], eps, beta, inv_n, eps_n);
+                if (REFRESH) vm.v[e] = m;
+            }
+            stf<VE, STREAM>(Th + o, vx);
+            stf<VE, STREAM>(ac + o, vc);
+            if (REFRESH) stf<VE, STREAM>(Mg + o, vm);
+            stf<VE, STREAM>(ib + o, vx);
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
+        float x = Th[j], acc = ac[j], m = REFRESH ? Mg[j] : 0.f;
+        delayed_nesterov<REFRESH>(x, m, acc, ob[j], eps, beta, inv_n, eps_n);
+        Th[j] = x;
+        ac[j] = acc;
+        if (REFRESH) Mg[j] = m;
+        ib[j] = x;
     }
 }
 

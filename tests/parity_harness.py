@@ -24,7 +24,8 @@ PER_EVENT_TOL = 1e-6   # max relative error per event (stated tolerance of the n
 FULL_TRACE_TOL = 1e-5  # after the full trace
 
 _BUF = {"Theta": hb.BUF_THETA_G, "Mg": hb.BUF_M_G, "th": hb.BUF_THETA_L, "ml": hb.BUF_M_L,
-        "anchor": hb.BUF_ANCHOR, "outbox": hb.BUF_OUTBOX, "inbox": hb.BUF_INBOX, "th0": hb.BUF_THETA0}
+        "anchor": hb.BUF_ANCHOR, "outbox": hb.BUF_OUTBOX, "inbox": hb.BUF_INBOX, "th0": hb.BUF_THETA0,
+        "acc": hb.BUF_ACC_L, "acc_g": hb.BUF_ACC_G}
 
 
 def rel_error(got: np.ndarray, want: np.ndarray) -> float:
@@ -93,6 +94,7 @@ class Lockstep:
                 pad = 1 if (input_mode == "ptrs_misaligned" and k % 2 == 1) else 0
                 buf = torch.empty(int(n) + pad + 8, dtype=wdt, device=device)
                 self.thH_parts.append(buf[pad:pad + int(n)])
+        self.delayed = hyper.get("optimizer", 0) == hb.OPT_DELAYED_NESTEROV
         self.inbox_iter = [0] * (max(worker_lps) + 1)
         self.log = []
         self.bit_identical = True
@@ -155,12 +157,12 @@ class Lockstep:
     def written_by(self, rec) -> List[Tuple[str, int]]:
         kind, l, w = rec["kind"], rec["lps"], rec["worker"]
         if kind == tr.ARRIVE:
-            out = [("th", l), ("ml", l), ("th0", w)]
+            out = [("th", l), ("ml", l), ("th0", w)] + ([("acc", l)] if self.delayed else [])
             if rec["pushed"]:
                 out.append(("outbox", l))
             return out
         if kind == tr.GPS_RECV:
-            return [("Theta", 0), ("Mg", 0), ("inbox", l)]
+            return [("Theta", 0), ("Mg", 0), ("inbox", l)] + ([("acc_g", 0)] if self.delayed else [])
         return [("th", l), ("anchor", l)]
 
     def all_buffers(self) -> List[Tuple[str, int]]:
@@ -169,6 +171,8 @@ class Lockstep:
         for l in range(n_lps):
             out += [(b, l) for b in ("th", "ml", "anchor", "outbox", "inbox")]
         out += [("th0", w) for w in range(len(self.worker_lps))]
+        if self.delayed:
+            out += [("acc_g", 0)] + [("acc", l) for l in range(n_lps)]
         return out
 
     # ------------------------------------------------------------------ comparison

@@ -500,3 +500,72 @@ def test_batched_replay_against_oracle_160m_window():
     ls.compare(ls.all_buffers(), FULL_TRACE_TOL)
     assert ls.bit_identical
     ls.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# optional delayed-Nesterov optimizer (the paper's experimental setting: d_l = 16, d_g = 2)
+# ---------------------------------------------------------------------------------------------
+DN_HP = dict(eta_l=3.2, beta_l=0.9, eta_g=0.3, beta_g=0.5, alpha=0.25, optimizer=hb.OPT_DELAYED_NESTEROV,
+             delay_l=16, delay_g=2)
+
+
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+@pytest.mark.parametrize("mode", ["flat", "ptrs_misaligned"])
+def test_delayed_nesterov_small_shapes(wdt, mode):
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 1])
+    worker_lps = [0, 0, 1, 1, 1]
+    hp = dict(DN_HP, K=5, delay_l=3)
+    events = tr.random_trace(worker_lps, 120, 5, seed=77)
+    ls = Lockstep(lay, worker_lps, hp, wdt, seed=6, chunk_elems=1024, input_mode=mode)
+    ls.run(events, check_every=1, full_check_every=30)
+    assert ls.bit_identical and ls.max_err == 0.0
+    assert ls.h.counters(0)["i"] >= 4
+    ls.close()
+
+
+def test_delayed_nesterov_toy_config_paper_settings():
+    wl = workloads.workload("toy_k4")
+    hp = dict(DN_HP, K=wl.K)
+    ls = Lockstep(wl.layout, wl.worker_lps, hp, wl.worker_dtype, wl.seed)
+    ls.run(wl.trace(), check_every=1, full_check_every=100)
+    assert ls.bit_identical and ls.max_err <= PER_EVENT_TOL
+    ls.close()
+
+
+def test_delayed_nesterov_replay_and_checkpoint(tmp_path):
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.decoder_layout("tiny", 2, 64, 300)
+    worker_lps = [0, 0, 1, 1]
+    hp = dict(DN_HP, K=4, delay_l=3)
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=[1.0, 2.5, 3.0, 1.7],
+                                            t_profiled_ms=1.0, n_arrivals=90, K=4))
+    dg = DeviceGenerator(lay, 19)
+    bufs = [torch.empty(lay.P, dtype=torch.float32, device="cuda") for _ in worker_lps]
+
+    def run(h, evs, mb):
+        def producer(index, worker, rnd):
+            return dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker])
+        return h.replay(evs, producer, max_batch=mb)
+
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, **hp)
+    run(ref, events, 1)
+    a = hb.Halos(dg.theta_init(), worker_lps, lay.numel, **hp)
+    run(a, events[:37], 4)                 # batching requested: this optimizer still launches event by event
+    assert a.batch_info()["multi_launches"] == 0
+    a.export_file(tmp_path / "dn.ckpt")
+    a.close()
+    b = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, **hp)
+    b.import_file(tmp_path / "dn.ckpt")
+    run(b, events[37:], 1)
+    for which in (hb.BUF_THETA_G, hb.BUF_M_G, hb.BUF_ACC_G):
+        assert np.array_equal(ref.read(which).view(np.uint32), b.read(which).view(np.uint32))
+    for l in (0, 1):
+        for which in (hb.BUF_THETA_L, hb.BUF_M_L, hb.BUF_ACC_L, hb.BUF_ANCHOR):
+            assert np.array_equal(ref.read(which, l).view(np.uint32), b.read(which, l).view(np.uint32))
+    plain = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, K=4)
+    with pytest.raises(hb.HalosError):
+        plain.import_file(tmp_path / "dn.ckpt")       # other optimizer: refused
+    with pytest.raises(hb.HalosError):
+        plain.read(hb.BUF_ACC_G)
+    for h in (ref, b, plain):
+        h.close()
