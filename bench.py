@@ -445,6 +445,8 @@ def main():
         d_bytes = kernel_bytes(dominant, dn) / dn
         achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
         tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
+        if dominant == "arrive_multi" and wname == "f32" and n_multi:
+            tpp = 15.24 + 12.0 * n_batched / n_multi     # measured: model and momentum cross HBM once per batch
         roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak,
                     "unit": "GB/s", "frac": achieved / peak, "traffic": (tpp * P if tpp else None),
                     "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel}
