@@ -45,8 +45,9 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {"arrive_f32": 28, "arrive_bf16": 22, "arrive_push_f32": 36, "arrive_push_bf16": 30,
                    "push": 12, "gps": 24, "pull": 16}
 
-# DRAM read+write bytes per parameter per launch from the ncu capture summarised in
-# profiles/ncu_full_kernels_70m_f32_small.md (P = 70,426,624; traffic is proportional to P).
+# DRAM read+write bytes per parameter per launch, from an ncu capture of the 70M-parameter fp32
+# profiling workload (P = 70,426,624; the summary is kept with the other ncu summaries; traffic is
+# proportional to P).
 DRAM_BYTES_PER_PARAM = {"arrive_f32": 27.22, "arrive_push_f32": 35.23, "gps": 23.20, "pull": 15.20}
 
 
@@ -270,7 +271,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--chunk-elems", type=int, default=0)
-    ap.add_argument("--max-batch", type=int, default=4,
+    ap.add_argument("--max-batch", type=int, default=8,
                     help="multi-event fusion in the driver: up to this many arrivals per launch (1 = one kernel per event)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over buffer sizes instead of the default line")
     ap.add_argument("--sweep-max", type=int, default=0, help="largest size to include (0 = all)")

@@ -61,7 +61,8 @@ enum { HALOS_OPT_PAPER = 0, HALOS_OPT_DELAYED_NESTEROV = 1 };
 
 /* flags */
 enum {
-    HALOS_FLAG_STATS = 1u          /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
+    HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
+    HALOS_FLAG_GUARD = 2u          /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
 };
 
 /* LPS phase of the push / merge round trip */
@@ -194,7 +195,7 @@ typedef int (*halos_producer_fn)(void* user, uint32_t event_index, uint32_t work
 int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                  void* user, halos_event_log* log_host, uint32_t* failed_at);
 
-/* The same replay with multi-event fusion: up to max_batch (<= 4) arrivals at one LPS, from distinct
+/* The same replay with multi-event fusion: up to max_batch (<= 8) arrivals at one LPS, from distinct
  * workers, are applied by ONE kernel that reads and writes that LPS's model and momentum once for
  * the whole batch (per element the updates are applied in queue order, so the state after the call
  * is bit-identical to halos_replay, and so is the log except for its `fused` flags).  Counters, the
@@ -239,6 +240,12 @@ int halos_info(halos_ctx* ctx, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chu
 int halos_export_file(halos_ctx* ctx, const char* path);
 int halos_import_file(halos_ctx* ctx, const char* path);
 
+/* Out-of-bounds write detector for test runs (needs HALOS_FLAG_GUARD): waits for the stream and checks
+ * the canary bytes around every state buffer.  *first_bad = -1 if all are intact, else the index of the
+ * first damaged buffer in allocation order (Theta, m_g, [acc_g], then per LPS theta, m_l, anchor, outbox,
+ * inbox, [acc], then the worker snapshots). */
+int halos_check_guards(halos_ctx* ctx, int32_t* first_bad);
+
 /* Multi-event fusion counters since creation: launches of the multi-arrival kernel and the number
  * of arrivals they covered (algorithmic bytes of those launches: (16 launches + 3 w_b arrivals) P). */
 int halos_batch_info(halos_ctx* ctx, uint64_t* multi_launches, uint64_t* batched_arrivals);
@@ -252,7 +259,7 @@ enum {
     HALOS_K_PUSH = 2,
     HALOS_K_GPS = 3,          /* global momentum update + Theta_i snapshot */
     HALOS_K_PULL = 4,         /* merge + anchor reset */
-    HALOS_K_ARRIVE_MULTI = 5, /* 2-4 arrivals at one LPS in one pass (halos_replay_batched) */
+    HALOS_K_ARRIVE_MULTI = 5, /* 2-8 arrivals at one LPS in one pass (halos_replay_batched) */
     HALOS_K_COUNT = 6
 };
 int halos_timing_enable(halos_ctx* ctx, int on);

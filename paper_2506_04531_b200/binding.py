@@ -21,6 +21,7 @@ LIB_PATH = Path(os.environ.get("HALOS_B200_LIB", _PKG / "libhalos_b200.so"))
 OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED = range(6)
 F32, BF16 = 0, 1
 FLAG_STATS = 1
+FLAG_GUARD = 2
 IDLE, PUSHED, ANSWERED = 0, 1, 2
 BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0, BUF_ACC_L, BUF_ACC_G = range(10)
 OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1
@@ -33,7 +34,7 @@ EXPORTED = (
     "halos_lps_push", "halos_gps_merge", "halos_lps_pull", "halos_destroy", "halos_replay", "halos_peek",
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
     "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
-    "halos_import_file", "halos_replay_batched", "halos_batch_info",
+    "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -99,6 +100,7 @@ def load_library():
     lib.halos_destroy.argtypes = [vp]
     lib.halos_replay.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32)]
     lib.halos_replay_batched.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
+    lib.halos_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.halos_batch_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
     lib.halos_peek.argtypes = [vp, u32, u32, C.POINTER(vp), C.POINTER(u64)]
     lib.halos_read.argtypes = [vp, u32, u32, u64, u64, vp]
@@ -358,6 +360,12 @@ class Halos:
 
     def import_file(self, path):
         self._check(self._lib.halos_import_file(self._h, str(path).encode()))
+
+    def check_guards(self) -> int:
+        """-1 if every canary zone is intact, else the index of the first damaged buffer (FLAG_GUARD contexts)."""
+        bad = C.c_int32(0)
+        self._check(self._lib.halos_check_guards(self._h, C.byref(bad)))
+        return int(bad.value)
 
     def batch_info(self) -> dict:
         a, b = C.c_uint64(), C.c_uint64()

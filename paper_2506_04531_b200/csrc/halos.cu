@@ -43,6 +43,13 @@ struct WorkerState {
     cudaEvent_t table_copied = nullptr;  // guards reuse of the pinned pointer-table slot
 };
 
+constexpr size_t kGuardBytes = 256;
+struct GuardedBuffer {
+    char* raw;       // start of the allocation: [guard | data (bytes) | slack + guard]
+    size_t padded;   // data size rounded up to 256
+    size_t bytes;    // data size
+};
+
 struct TimedLaunch {
     cudaEvent_t a, b;
     int kind;
@@ -82,6 +89,7 @@ struct halos_ctx {
     int stage_next = 0;
 
     std::vector<void*> owned;  // device allocations made through the allocator
+    std::vector<GuardedBuffer> guards;
     uint64_t launches = 0;
     uint64_t batched_arrivals = 0;  // arrivals that ran inside a multi-arrival launch
     uint64_t multi_launches = 0;
@@ -359,10 +367,11 @@ int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push)
     a.eta = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.omb = 1.0f - c->cfg.beta_l;
-    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
+    const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     Timer tm(c, HALOS_K_ARRIVE_MULTI);
-    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-    else arrive_multi_kernel<W, NB, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    else arrive_multi_kernel<W, NB, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
     tm.stop();
     c->launches++;
     c->batched_arrivals += NB;
@@ -382,6 +391,10 @@ int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool 
         case 2: rc = launch_arrive_multi<W, 2>(c, s, q.data(), push); break;
         case 3: rc = launch_arrive_multi<W, 3>(c, s, q.data(), push); break;
         case 4: rc = launch_arrive_multi<W, 4>(c, s, q.data(), push); break;
+        case 5: rc = launch_arrive_multi<W, 5>(c, s, q.data(), push); break;
+        case 6: rc = launch_arrive_multi<W, 6>(c, s, q.data(), push); break;
+        case 7: rc = launch_arrive_multi<W, 7>(c, s, q.data(), push); break;
+        case 8: rc = launch_arrive_multi<W, 8>(c, s, q.data(), push); break;
         default: rc = fail(c, HALOS_ERR_INVALID_ARG, "internal: batch larger than %d", kMaxBatch);
     }
     q.clear();
@@ -478,6 +491,16 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     CUC(cudaSetDevice(cfg->device));
     const size_t P = c->P, nt = cfg->n_tensors, nc = c->chunks.size();
     auto A = [&](size_t bytes) { return dev_alloc(c, bytes); };
+    // State buffers: with HALOS_FLAG_GUARD each gets a 256-byte canary zone on both sides.
+    const bool guard = (cfg->flags & HALOS_FLAG_GUARD) != 0;
+    auto S = [&](size_t bytes) -> void* {
+        if (!guard) return dev_alloc(c, bytes);
+        const size_t padded = (bytes + 255) / 256 * 256;
+        char* raw = (char*)dev_alloc(c, padded + 2 * kGuardBytes);
+        if (!raw) return nullptr;
+        c->guards.push_back(GuardedBuffer{raw, padded, bytes});
+        return raw + kGuardBytes;
+    };
     bool ok = true;
     ok &= (c->d_chunks = (Chunk*)A(nc * sizeof(Chunk))) != nullptr;
     ok &= (c->d_tensor_off = (unsigned long long*)A((nt + 1) * 8)) != nullptr;
@@ -488,26 +511,30 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
         ok &= (c->d_partial_Delta = (double*)A(nc * 8)) != nullptr;
         ok &= (c->d_stats = (double*)A((size_t)2 * cfg->n_lps * nt * 8)) != nullptr;
     }
-    ok &= (c->Theta = (float*)A(P * 4)) != nullptr;
-    ok &= (c->Mg = (float*)A(P * 4)) != nullptr;
+    ok &= (c->Theta = (float*)S(P * 4)) != nullptr;
+    ok &= (c->Mg = (float*)S(P * 4)) != nullptr;
     const bool dn = cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV;
-    if (dn) ok &= (c->acc_g = (float*)A(P * 4)) != nullptr;
+    if (dn) ok &= (c->acc_g = (float*)S(P * 4)) != nullptr;
     c->lps.resize(cfg->n_lps);
     for (auto& s : c->lps) {
         if (!ok) break;
-        ok &= (s.th = (float*)A(P * 4)) != nullptr;
-        ok &= (s.ml = (float*)A(P * 4)) != nullptr;
-        ok &= (s.anchor = (float*)A(P * 4)) != nullptr;
-        ok &= (s.outbox = (float*)A(P * 4)) != nullptr;
-        ok &= (s.inbox = (float*)A(P * 4)) != nullptr;
-        if (dn) ok &= (s.acc = (float*)A(P * 4)) != nullptr;
+        ok &= (s.th = (float*)S(P * 4)) != nullptr;
+        ok &= (s.ml = (float*)S(P * 4)) != nullptr;
+        ok &= (s.anchor = (float*)S(P * 4)) != nullptr;
+        ok &= (s.outbox = (float*)S(P * 4)) != nullptr;
+        ok &= (s.inbox = (float*)S(P * 4)) != nullptr;
+        if (dn) ok &= (s.acc = (float*)S(P * 4)) != nullptr;
     }
     c->workers.resize(cfg->n_workers);
     for (uint32_t w = 0; w < cfg->n_workers && ok; ++w) {
         c->workers[w].lps = c->worker_lps[w];
-        ok &= (c->workers[w].th0 = A(P * c->wb)) != nullptr;
+        ok &= (c->workers[w].th0 = S(P * c->wb)) != nullptr;
     }
     if (!ok) return bail(HALOS_ERR_OOM, "device allocation failed");
+    for (auto& g : c->guards) {   // canaries: 0xA5 before the data, and from the end of the data to the end of the block
+        CUC(cudaMemsetAsync(g.raw, 0xA5, kGuardBytes, c->stream));
+        CUC(cudaMemsetAsync(g.raw + kGuardBytes + g.bytes, 0xA5, g.padded - g.bytes + kGuardBytes, c->stream));
+    }
     for (void* p : c->owned)
         if (reinterpret_cast<uintptr_t>(p) & 255) return bail(HALOS_ERR_INVALID_ARG, "allocator returned a pointer not aligned to 256 bytes");
 
@@ -980,6 +1007,29 @@ int halos_info(halos_ctx* c, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunk
     if (n_tensors) *n_tensors = (uint32_t)c->tensor_numel.size();
     if (n_chunks) *n_chunks = (uint32_t)c->chunks.size();
     if (launches) *launches = c->launches;
+    return HALOS_OK;
+}
+
+int halos_check_guards(halos_ctx* c, int32_t* first_bad) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (!(c->cfg.flags & HALOS_FLAG_GUARD)) return fail(c, HALOS_ERR_BAD_STATE, "context was created without HALOS_FLAG_GUARD");
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->stream));
+    int32_t bad = -1;
+    std::vector<unsigned char> host;
+    for (size_t k = 0; k < c->guards.size() && bad < 0; ++k) {
+        const GuardedBuffer& g = c->guards[k];
+        const size_t tail = g.padded - g.bytes + kGuardBytes;
+        host.resize(kGuardBytes + tail);
+        CU(c, cudaMemcpy(host.data(), g.raw, kGuardBytes, cudaMemcpyDeviceToHost));
+        CU(c, cudaMemcpy(host.data() + kGuardBytes, g.raw + kGuardBytes + g.bytes, tail, cudaMemcpyDeviceToHost));
+        for (unsigned char b : host)
+            if (b != 0xA5) {
+                bad = (int32_t)k;
+                break;
+            }
+    }
+    if (first_bad) *first_bad = bad;
     return HALOS_OK;
 }
 

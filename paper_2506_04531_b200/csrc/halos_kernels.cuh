@@ -343,9 +343,11 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
 // and momentum are read and written once for the whole batch; per element the NB updates are applied
 // in queue order in registers, so the result is bit-identical to NB single launches.  Traffic per
 // batch: 8 + 8 (theta, m read + write) + NB x (2 w_b read + w_b write) instead of NB x (16 + 3 w_b).
-// Only the last arrival of a batch may close a window of K (PUSH).
+// Only the last arrival of a batch may close a window of K (PUSH).  Batches of up to 4 run with the
+// regular CTA size; 5..8 need ~150 registers per thread and run with 256-thread CTAs.
 // =====================================================================================================
-constexpr int kMaxBatch = 4;
+constexpr int kMaxBatch = 8;
+constexpr int kMultiWideThreads = 256;   // CTA size of the multi-arrival kernel for batches of 3..8 (register budget)
 
 template <class W>
 struct ArriveMultiArgs {
@@ -360,8 +362,8 @@ struct ArriveMultiArgs {
     float eta, beta, omb;
 };
 
-template <class W, int NB, bool PUSH, bool STREAM, int VE>
-__global__ void __launch_bounds__(kThreads, (NB <= 2 ? 1024 / kThreads : 1))
+template <class W, int NB, bool PUSH, bool STREAM, int VE, int TPB>
+__global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
 arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
     using T = WTraits<W>;
     const Chunk c = chunks[blockIdx.x];
@@ -382,7 +384,7 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
     uint32_t done = 0;
     if (vec_ok) {
         const uint32_t nvec = c.count / VE;
-        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+        for (uint32_t v = threadIdx.x; v < nvec; v += TPB) {
             const size_t o = (size_t)VE * v;
             FVec<VE> vh[NB], vs[NB], vx, vm, va;
 #pragma unroll
@@ -413,7 +415,7 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
         }
         done = nvec * VE;
     }
-    for (uint32_t i = done + threadIdx.x; i < c.count; i += kThreads) {
+    for (uint32_t i = done + threadIdx.x; i < c.count; i += TPB) {
         float x = th[i], m = ml[i];
 #pragma unroll
         for (int j = 0; j < NB; ++j) {

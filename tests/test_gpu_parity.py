@@ -115,9 +115,11 @@ def test_small_shapes_bit_exact(shape, wdt, mode):
     worker_lps = [0, 0, 1, 1, 1]
     events = tr.random_trace(worker_lps, 60, 3, seed=zlib.crc32(f"{shape}/{wdt}/{mode}".encode()) & 0xFFFF)
     chunk = 1024 if shape in ("ragged_big", "p4097") else 0
-    ls = Lockstep(lay, worker_lps, dict(K=3, **PAPER_HP), wdt, seed=5, chunk_elems=chunk, input_mode=mode)
+    ls = Lockstep(lay, worker_lps, dict(K=3, **PAPER_HP), wdt, seed=5, chunk_elems=chunk, input_mode=mode,
+                  flags=hb.FLAG_GUARD)
     ls.run(events, check_every=1, full_check_every=20)
     assert ls.bit_identical and ls.max_err == 0.0
+    assert ls.h.check_guards() == -1          # no kernel wrote outside its buffers
     ls.close()
 
 
@@ -430,15 +432,15 @@ def test_out_of_memory_is_reported_and_cleaned_up():
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
 @pytest.mark.parametrize("mode", ["flat", "ptrs"])
-@pytest.mark.parametrize("max_batch", [2, 3, 4, 9])
+@pytest.mark.parametrize("max_batch", [2, 3, 4, 6, 8, 99])
 def test_batched_replay_is_bit_identical(wdt, mode, max_batch):
     from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
     lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 3])
-    worker_lps = [0, 0, 0, 0, 0, 1, 1, 1, 2]
-    hp = dict(K=5, **PAPER_HP)
-    speeds = [1.0, 2.5, 3.0, 1.7, 3.9, 1.1, 1.2, 3.3, 2.0]
+    worker_lps = [0, 0, 0, 0, 0, 0, 0, 0, 1, 1, 1, 2]
+    hp = dict(K=11, **PAPER_HP)
+    speeds = [1.0, 1.05, 1.1, 1.15, 1.2, 1.25, 1.3, 3.9, 1.1, 1.2, 3.3, 2.0]
     events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=speeds, t_profiled_ms=1.0,
-                                            n_arrivals=260, K=5))
+                                            n_arrivals=300, K=11))
     dg = DeviceGenerator(lay, 23)
     tdt = torch.float32 if wdt == gen.F32 else torch.int16
     off = lay.offsets.astype(np.int64)
@@ -569,3 +571,21 @@ def test_delayed_nesterov_replay_and_checkpoint(tmp_path):
         plain.read(hb.BUF_ACC_G)
     for h in (ref, b, plain):
         h.close()
+
+
+def test_guard_zones_detect_an_out_of_bounds_write():
+    P = 1001                                   # odd size: the tail guard starts right after the last element
+    h = hb.Halos(torch.zeros(P, device="cuda"), [0], flags=hb.FLAG_GUARD)
+    assert h.check_guards() == -1
+    th = h.peek(hb.BUF_THETA_L, 0)
+    # simulate a stray write one element past the end of theta (3rd state buffer: Theta, m_g, theta_0)
+    end_addr = th.data_ptr() + 4 * P
+    iface = {"shape": (1,), "typestr": "<f4", "data": (end_addr, False), "version": 2}
+    holder = type("_Mem", (), {"__cuda_array_interface__": iface})()
+    torch.as_tensor(holder, device="cuda").fill_(1.0)
+    assert h.check_guards() == 2
+    h.close()
+    plain = hb.Halos(torch.zeros(8, device="cuda"), [0])
+    with pytest.raises(hb.HalosError):
+        plain.check_guards()
+    plain.close()
