@@ -24,6 +24,8 @@ def test_window_events_and_oracle_sample():
     assert len(ev2) == 1280 and np.array_equal(ev2[:200], ev[:200])
     rate, desc, spent, done = bench.oracle_sample(wl, ev[:40], 1 << 14, budget_s=5.0)
     assert done == 40 and rate > 1e5 and "index slice" in desc
+    all_rate, cores = bench.oracle_sample_all_cores(wl, ev[:40], 1 << 14, budget_s=5.0)
+    assert cores >= 1 and all_rate > 1e5
 
 
 def _rank_main(rank, world, port, out_dir):
