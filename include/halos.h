@@ -62,7 +62,10 @@ enum { HALOS_OPT_PAPER = 0, HALOS_OPT_DELAYED_NESTEROV = 1 };
 /* flags */
 enum {
     HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
-    HALOS_FLAG_GUARD = 2u          /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
+    HALOS_FLAG_GUARD = 2u,         /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
+    HALOS_FLAG_MATERIALISE_DELTA = 4u  /* halos_worker_delta forms delta (fp32) into a context buffer at once, so the
+                                          borrow of theta_H ends when that call has been enqueued; costs one 4P
+                                          buffer per worker and 4 + 2 w_b extra bytes of traffic per parameter */
 };
 
 /* LPS phase of the push / merge round trip */
@@ -121,8 +124,10 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
  * delta never touches memory.  Exactly one of thetaH_flat_dev (device, P elements of worker_dtype,
  * packed like the state) and thetaH_ptrs_host (host array of n_tensors DEVICE pointers, one per
  * tensor, each tensor contiguous) is non-NULL.  The device data is BORROWED until the matching
- * halos_lps_apply has completed in stream order.  BAD_STATE if the worker already has a pending
- * result. */
+ * halos_lps_apply has completed in stream order -- or, on a context created with
+ * HALOS_FLAG_MATERIALISE_DELTA, only until the work this call enqueues has completed (delta is then
+ * written to a context buffer by a kernel of its own and halos_lps_apply reads that buffer; the
+ * resulting state is bit-identical).  BAD_STATE if the worker already has a pending result. */
 int halos_worker_delta(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_dev,
                        const void* const* thetaH_ptrs_host);
 
@@ -243,7 +248,7 @@ int halos_import_file(halos_ctx* ctx, const char* path);
 /* Out-of-bounds write detector for test runs (needs HALOS_FLAG_GUARD): waits for the stream and checks
  * the canary bytes around every state buffer.  *first_bad = -1 if all are intact, else the index of the
  * first damaged buffer in allocation order (Theta, m_g, [acc_g], then per LPS theta, m_l, anchor, outbox,
- * inbox, [acc], then the worker snapshots). */
+ * inbox, [acc], then per worker its snapshot [and its materialised delta]). */
 int halos_check_guards(halos_ctx* ctx, int32_t* first_bad);
 
 /* Multi-event fusion counters since creation: launches of the multi-arrival kernel and the number

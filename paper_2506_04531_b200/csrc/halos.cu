@@ -30,10 +30,11 @@ struct LpsState {
     int phase = HALOS_IDLE;
 };
 
-enum { PEND_NONE = 0, PEND_FLAT = 1, PEND_PTRS = 2, PEND_STAGED = 3 };
+enum { PEND_NONE = 0, PEND_FLAT = 1, PEND_PTRS = 2, PEND_STAGED = 3, PEND_DELTA = 4 };
 
 struct WorkerState {
     void* th0 = nullptr;
+    float* delta = nullptr;  // materialised displacement (HALOS_FLAG_MATERIALISE_DELTA only)
     uint32_t lps = 0;
     int pending = PEND_NONE;
     const void* flat = nullptr;
@@ -243,6 +244,18 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
 template <class W>
 int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
     if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat);
+    if (w.pending == PEND_DELTA) {
+        ArriveDeltaArgs<W> d{w.delta, (W*)w.th0, s.th, s.ml, s.anchor, s.outbox, c->cfg.eta_l, c->cfg.beta_l, 1.0f - c->cfg.beta_l};
+        const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+        if (grid.x == 0) return HALOS_OK;
+        Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+        if (push) arrive_delta_kernel<W, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, d);
+        else arrive_delta_kernel<W, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, d);
+        tm.stop();
+        c->launches++;
+        CU(c, cudaGetLastError());
+        return HALOS_OK;
+    }
     ArriveArgs<W> a;
     a.h_flat = (const W*)flat;
     a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)widx * c->tensor_numel.size());
@@ -282,6 +295,26 @@ int finalize_stats(halos_ctx* c, uint32_t what, uint32_t lps) {
     c->launches++;
     CU(c, cudaGetLastError());
     return HALOS_OK;
+}
+
+// delta[w] <- theta_H - theta0[w] now (Alg. 1 line 25 as a kernel of its own); flat == NULL: pointer table of w.
+template <class W>
+int launch_delta_t(halos_ctx* c, uint32_t worker, const void* flat) {
+    WorkerState& w = c->workers[worker];
+    DeltaArgs<W> a;
+    a.h_flat = (const W*)flat;
+    a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)worker * c->tensor_numel.size());
+    a.tensor_off = c->d_tensor_off;
+    a.th0 = (const W*)w.th0;
+    a.delta = w.delta;
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    if (grid.x) delta_kernel<W, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    c->launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+int launch_delta(halos_ctx* c, uint32_t worker, const void* flat) {
+    return c->wb == 4 ? launch_delta_t<float>(c, worker, flat) : launch_delta_t<uint16_t>(c, worker, flat);
 }
 
 // Host-side part of an arrival (Alg. 1 lines 10 and 13): argument/state checks and counter updates.
@@ -441,6 +474,9 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
         return fail(nullptr, HALOS_ERR_INVALID_ARG, "delays must be at least 1");
     if (cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV && (cfg->flags & HALOS_FLAG_STATS))
         return fail(nullptr, HALOS_ERR_UNSUPPORTED, "statistics are not available with the delayed Nesterov optimizer");
+    if ((cfg->flags & HALOS_FLAG_MATERIALISE_DELTA) &&
+        ((cfg->flags & HALOS_FLAG_STATS) || cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV))
+        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "materialised deltas combine neither with statistics nor with delayed Nesterov");
     if ((cfg->alloc == nullptr) != (cfg->free_ == nullptr)) return fail(nullptr, HALOS_ERR_INVALID_ARG, "alloc and free_ go together");
     for (uint32_t w = 0; w < cfg->n_workers; ++w)
         if (cfg->worker_lps[w] >= cfg->n_lps) return fail(nullptr, HALOS_ERR_INVALID_ARG, "worker_lps[%u] out of range", w);
@@ -529,6 +565,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     for (uint32_t w = 0; w < cfg->n_workers && ok; ++w) {
         c->workers[w].lps = c->worker_lps[w];
         ok &= (c->workers[w].th0 = S(P * c->wb)) != nullptr;
+        if (ok && (cfg->flags & HALOS_FLAG_MATERIALISE_DELTA)) ok &= (c->workers[w].delta = (float*)S(P * 4)) != nullptr;
     }
     if (!ok) return bail(HALOS_ERR_OOM, "device allocation failed");
     for (auto& g : c->guards) {   // canaries: 0xA5 before the data, and from the end of the data to the end of the block
@@ -593,6 +630,13 @@ int halos_worker_delta(halos_ctx* c, uint32_t worker, const void* flat, const vo
     if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u already has a pending result", worker);
     if (flat) {
         if (reinterpret_cast<uintptr_t>(flat) % c->wb) return fail(c, HALOS_ERR_INVALID_ARG, "thetaH not aligned to its element size");
+        if (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) {
+            CU(c, cudaSetDevice(c->cfg.device));
+            int rc = launch_delta(c, worker, flat);
+            if (rc != HALOS_OK) return rc;
+            w.pending = PEND_DELTA;
+            return HALOS_OK;
+        }
         w.flat = flat;
         w.pending = PEND_FLAT;
         return HALOS_OK;
@@ -608,6 +652,12 @@ int halos_worker_delta(halos_ctx* c, uint32_t worker, const void* flat, const vo
     std::memcpy(slot, ptrs, nt * 8);
     CU(c, cudaMemcpyAsync(c->d_ptr_tables + (size_t)worker * nt, slot, nt * 8, cudaMemcpyHostToDevice, c->stream));
     CU(c, cudaEventRecord(w.table_copied, c->stream));
+    if (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) {
+        int rc = launch_delta(c, worker, nullptr);
+        if (rc != HALOS_OK) return rc;
+        w.pending = PEND_DELTA;
+        return HALOS_OK;
+    }
     w.pending = PEND_PTRS;
     return HALOS_OK;
 }
@@ -636,6 +686,16 @@ int halos_worker_delta_host(halos_ctx* c, uint32_t worker, const void* host) {
     CU(c, cudaStreamWaitEvent(c->copy_stream, c->stage_free[slot], 0));
     CU(c, cudaMemcpyAsync(c->stage[slot], host, c->P * c->wb, cudaMemcpyHostToDevice, c->copy_stream));
     CU(c, cudaEventRecord(c->stage_ready[slot], c->copy_stream));
+    if (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) {
+        // delta is formed as soon as the copy has landed and the staging buffer is free again at once
+        CU(c, cudaStreamWaitEvent(c->stream, c->stage_ready[slot], 0));
+        int rc = launch_delta(c, worker, c->stage[slot]);
+        if (rc != HALOS_OK) return rc;
+        CU(c, cudaEventRecord(c->stage_free[slot], c->stream));
+        c->stage_next = (slot + 1) % kStageSlots;
+        w.pending = PEND_DELTA;
+        return HALOS_OK;
+    }
     c->stage_owner[slot] = (int)worker;
     c->stage_next = (slot + 1) % kStageSlots;
     w.slot = slot;
@@ -732,7 +792,8 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
     if (max_batch == 0) max_batch = 1;
     if (max_batch > (uint32_t)kMaxBatch) max_batch = kMaxBatch;
     if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
-    const bool immediate = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV;  // that optimizer is launched event by event
+    const bool immediate = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV ||       // launched event by event
+                           (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) != 0;
     std::vector<std::vector<Deferred>> queue(c->cfg.n_lps);
     int rc = HALOS_OK;
     uint32_t k = 0;

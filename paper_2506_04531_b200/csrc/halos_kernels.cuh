@@ -559,6 +559,105 @@ gps_dn_kernel(const Chunk* __restrict__ chunks, GpsDnArgs a) {
 }
 
 // =====================================================================================================
+// Materialised delta (HALOS_FLAG_MATERIALISE_DELTA): the worker-side subtraction of Alg. 1 line 25 runs
+// when the result is handed over, delta (fp32) is kept in a context buffer, and the caller's theta_H is
+// free again as soon as that kernel has been enqueued.  The LPS update then reads delta instead of
+// theta_H and the old snapshot.  Same roundings as the fused path, hence the same bits.
+// =====================================================================================================
+template <class W>
+struct DeltaArgs {
+    const W* h_flat;
+    const W* const* h_ptrs;
+    const unsigned long long* tensor_off;
+    const W* th0;
+    float* delta;
+};
+
+template <class W, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+delta_kernel(const Chunk* __restrict__ chunks, DeltaArgs<W> a) {
+    using T = WTraits<W>;
+    const Chunk c = chunks[blockIdx.x];
+    const W* h = a.h_flat ? a.h_flat + c.begin : a.h_ptrs[c.tensor] + (c.begin - a.tensor_off[c.tensor]);
+    const W* s0 = a.th0 + c.begin;
+    float* dl = a.delta + c.begin;
+    const bool vec_ok = ((c.begin % VE) == 0) && ((reinterpret_cast<uintptr_t>(h) % (VE * sizeof(W))) == 0);
+    uint32_t done = 0;
+    if (vec_ok) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vh = T::template load<VE, STREAM>(h + o);
+            FVec<VE> vs = T::template load<VE, STREAM>(s0 + o);
+            FVec<VE> d;
+#pragma unroll
+            for (int e = 0; e < VE; ++e) d.v[e] = __fsub_rn(vh.v[e], vs.v[e]);
+            stf<VE, STREAM>(dl + o, d);
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads)
+        dl[j] = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
+}
+
+template <class W>
+struct ArriveDeltaArgs {
+    const float* delta;
+    W* th0;
+    float* th;
+    float* ml;
+    const float* anchor;
+    float* outbox;
+    float eta, beta, omb;
+};
+
+template <class W, bool PUSH, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+arrive_delta_kernel(const Chunk* __restrict__ chunks, ArriveDeltaArgs<W> a) {
+    using T = WTraits<W>;
+    const Chunk c = chunks[blockIdx.x];
+    const float* dl = a.delta + c.begin;
+    W* s0 = a.th0 + c.begin;
+    float* th = a.th + c.begin;
+    float* ml = a.ml + c.begin;
+    const float* an = PUSH ? a.anchor + c.begin : nullptr;
+    float* ob = PUSH ? a.outbox + c.begin : nullptr;
+    const float eta = a.eta, beta = a.beta, omb = a.omb;
+    uint32_t done = 0;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vd = ldf<VE, STREAM>(dl + o);
+            FVec<VE> vx = ldf<VE, STREAM>(th + o);
+            FVec<VE> vm = ldf<VE, STREAM>(ml + o);
+            FVec<VE> va;
+            if (PUSH) va = ldf<VE, STREAM>(an + o);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) model_update(vx.v[e], vm.v[e], vd.v[e], eta, beta, omb);
+            stf<VE, STREAM>(th + o, vx);
+            stf<VE, STREAM>(ml + o, vm);
+            T::template store<VE, STREAM>(s0 + o, vx);
+            if (PUSH) {
+                FVec<VE> D;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                stf<VE, STREAM>(ob + o, D);
+            }
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
+        float x = th[j], m = ml[j];
+        model_update(x, m, dl[j], eta, beta, omb);
+        th[j] = x;
+        ml[j] = m;
+        T::store1(s0 + j, x);
+        if (PUSH) ob[j] = __fsub_rn(x, an[j]);
+    }
+}
+
+// =====================================================================================================
 // PUSH alone: Delta = theta_t - theta_{t_last}                                   Alg. 1 line 14
 // =====================================================================================================
 struct PushArgs {

@@ -589,3 +589,58 @@ def test_guard_zones_detect_an_out_of_bounds_write():
     with pytest.raises(hb.HalosError):
         plain.check_guards()
     plain.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# materialised deltas: the borrow of theta_H ends when halos_worker_delta has been enqueued
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+@pytest.mark.parametrize("mode", ["flat", "ptrs_misaligned"])
+def test_materialised_delta_matches_oracle(wdt, mode):
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 1])
+    worker_lps = [0, 0, 1, 1, 1]
+    events = tr.random_trace(worker_lps, 90, 4, seed=55)
+    ls = Lockstep(lay, worker_lps, dict(K=4, **PAPER_HP), wdt, seed=12, chunk_elems=1024, input_mode=mode,
+                  flags=hb.FLAG_MATERIALISE_DELTA | hb.FLAG_GUARD)
+    ls.run(events, check_every=1, full_check_every=30)
+    assert ls.bit_identical and ls.max_err == 0.0 and ls.h.check_guards() == -1
+    ls.close()
+
+
+def test_materialised_delta_frees_the_callers_buffer():
+    from oracle import HalosOracle
+    lay = layouts.flat_layout("x", 100_003)
+    init = gen.theta_init(lay, 9)
+    h = hb.Halos(torch.from_numpy(init).cuda(), [0, 0, 0], K=3, flags=hb.FLAG_MATERIALISE_DELTA, **PAPER_HP)
+    o = HalosOracle(init, [0, 0, 0], K=3, **PAPER_HP)
+    scratch = torch.empty(lay.P, device="cuda")
+    pinned = torch.empty(lay.P).pin_memory()
+    for rnd in range(3):
+        results = [gen.worker_result(o.buffer("th0", w), lay, 9, w, rnd) for w in range(3)]
+        # all three results pass through ONE device buffer (and one pinned host buffer): each is overwritten
+        # by the next before any of them has been applied
+        scratch.copy_(torch.from_numpy(results[0]))
+        h.worker_delta(0, scratch)
+        scratch.copy_(torch.from_numpy(results[1]))
+        h.worker_delta(1, scratch)
+        pinned.copy_(torch.from_numpy(results[2]))
+        h.worker_delta_host(2, pinned)
+        torch.cuda.synchronize()
+        pinned.zero_()
+        scratch.zero_()
+        for w in (1, 2, 0):
+            due = h.lps_apply(0, w)
+            assert due == o.arrive(w, results[w])
+            if due:
+                h.lps_push(0)
+                h.gps_merge(0)
+                o.gps_recv(0)
+                h.lps_pull(0)
+                o.pull(0)
+    for which, name in ((hb.BUF_THETA_L, "th"), (hb.BUF_M_L, "ml"), (hb.BUF_ANCHOR, "anchor")):
+        assert np.array_equal(h.read(which, 0).view(np.uint32), o.buffer(name, 0).view(np.uint32))
+    assert np.array_equal(h.read(hb.BUF_THETA_G).view(np.uint32), o.buffer("Theta").view(np.uint32))
+    h.close()
+    with pytest.raises(hb.HalosError) as e:
+        hb.Halos(torch.zeros(8, device="cuda"), [0], flags=hb.FLAG_MATERIALISE_DELTA | hb.FLAG_STATS)
+    assert e.value.status == hb.ERR_UNSUPPORTED
