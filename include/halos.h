@@ -61,7 +61,7 @@ enum { HALOS_OPT_PAPER = 0, HALOS_OPT_DELAYED_NESTEROV = 1 };
 
 /* flags */
 enum {
-    HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta (arrive) and Delta (push) */
+    HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta, theta_t (arrive) and Delta (push) */
     HALOS_FLAG_GUARD = 2u,         /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
     HALOS_FLAG_MATERIALISE_DELTA = 4u  /* halos_worker_delta forms delta (fp32) into a context buffer at once, so the
                                           borrow of theta_H ends when that call has been enqueued; costs one 4P
@@ -228,8 +228,8 @@ int halos_counters(halos_ctx* ctx, uint32_t lps, uint64_t* counters_host);
 int halos_worker_info(halos_ctx* ctx, uint32_t worker, uint64_t* info_host);
 
 /* Per-tensor squared norms (needs HALOS_FLAG_STATS): what = 0: sum delta^2 of the last
- * halos_lps_apply of this LPS; what = 1: sum Delta^2 of its last halos_lps_push.  Waits for the
- * stream.  out_host: [n_tensors] doubles. */
+ * halos_lps_apply of this LPS; what = 1: sum Delta^2 of its last halos_lps_push; what = 2: sum theta_t^2 of
+ * its model right after that last halos_lps_apply.  Waits for the stream.  out_host: [n_tensors] doubles. */
 int halos_stats(halos_ctx* ctx, uint32_t what, uint32_t lps, double* out_host);
 
 /* Number of parameters P, tensors, scheduler chunks, and kernels launched so far. */

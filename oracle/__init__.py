@@ -63,6 +63,7 @@ def _load():
     lib.halos_oracle_error.argtypes = [c.c_void_p]
     lib.halos_oracle_arrive.argtypes = [c.c_void_p, c.c_uint32, c.c_void_p, c.POINTER(c.c_int)]
     lib.halos_oracle_gps_recv.argtypes = [c.c_void_p, c.c_uint32]
+    lib.halos_oracle_push.argtypes = [c.c_void_p, c.c_uint32]
     lib.halos_oracle_pull.argtypes = [c.c_void_p, c.c_uint32]
     lib.halos_oracle_buffer.restype = c.c_void_p
     lib.halos_oracle_buffer.argtypes = [c.c_void_p, c.c_int, c.c_uint32]
@@ -146,6 +147,10 @@ class HalosOracle:
         pushed = ctypes.c_int(0)
         self._check(self._lib.halos_oracle_arrive(self._h, int(worker), a.ctypes.data, ctypes.byref(pushed)))
         return bool(pushed.value)
+
+    def push(self, lps: int) -> None:
+        """Form Delta = theta_t - theta_{t_last} now (line 14), whatever the window counter says."""
+        self._check(self._lib.halos_oracle_push(self._h, int(lps)))
 
     def gps_recv(self, lps: int) -> None:
         """The GPS receives Delta from this LPS and answers with Theta_i (lines 2-4)."""

@@ -88,6 +88,11 @@ int halos_oracle_arrive(void* hv, uint32_t w, const void* thetaH, int* pushed) {
         if (pushed) *pushed = p ? 1 : 0;
     });
 }
+// Alg. 1 line 14 on its own (tests that push at times other than the window of K)
+int halos_oracle_push(void* hv, uint32_t l) {
+    Handle* h = (Handle*)hv;
+    return guarded(h, [&] { h->is_double ? h->d->push(l) : h->f->push(l); });
+}
 int halos_oracle_gps_recv(void* hv, uint32_t l) {
     Handle* h = (Handle*)hv;
     return guarded(h, [&] { h->is_double ? h->d->gps_recv(l) : h->f->gps_recv(l); });

@@ -255,16 +255,16 @@ class Halos:
         thetaH_ptrs: one CUDA tensor (or address) per layout tensor."""
         if thetaH_ptrs is not None:
             arr = (C.c_void_p * self.n_tensors)(*[_ptr(t) for t in thetaH_ptrs])
-            self._keep[worker] = (thetaH_ptrs, arr)
             self._check(self._lib.halos_worker_delta(self._h, worker, None, arr))
+            self._keep[worker] = (thetaH_ptrs, arr)      # borrowed until the apply: keep the tensors alive
         else:
-            self._keep[worker] = thetaH
             self._check(self._lib.halos_worker_delta(self._h, worker, _ptr(thetaH), None))
+            self._keep[worker] = thetaH
 
     def worker_delta_host(self, worker: int, thetaH_host):
         """thetaH_host: flat host tensor/array in the worker dtype (pinned memory makes the copy asynchronous)."""
-        self._keep[worker] = thetaH_host
         self._check(self._lib.halos_worker_delta_host(self._h, worker, _ptr(thetaH_host)))
+        self._keep[worker] = thetaH_host
 
     def lps_apply(self, lps: int, worker: int) -> bool:
         due = C.c_int(0)

@@ -74,8 +74,8 @@ struct halos_ctx {
     uint32_t* d_tensor_chunk_begin = nullptr;
     const void** d_ptr_tables = nullptr;  // [n_workers][n_tensors]
     const void** h_ptr_tables = nullptr;  // pinned mirror
-    double *d_partial_delta = nullptr, *d_partial_Delta = nullptr;
-    double* d_stats = nullptr;  // [2][n_lps][n_tensors]
+    double *d_partial_delta = nullptr, *d_partial_Delta = nullptr, *d_partial_theta = nullptr;
+    double* d_stats = nullptr;  // [3][n_lps][n_tensors]
 
     float *Theta = nullptr, *Mg = nullptr;
     float* acc_g = nullptr;  // delayed Nesterov only
@@ -267,6 +267,7 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
     a.outbox = s.outbox;
     a.partial_delta = c->d_partial_delta;
     a.partial_Delta = c->d_partial_Delta;
+    a.partial_theta = c->d_partial_theta;
     a.eta = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.omb = 1.0f - c->cfg.beta_l;
@@ -290,7 +291,7 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
 int finalize_stats(halos_ctx* c, uint32_t what, uint32_t lps) {
     const uint32_t nt = (uint32_t)c->tensor_numel.size();
     double* out = c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt;
-    const double* partial = what == 0 ? c->d_partial_delta : c->d_partial_Delta;
+    const double* partial = what == 0 ? c->d_partial_delta : what == 1 ? c->d_partial_Delta : c->d_partial_theta;
     stats_finalize_kernel<<<nt, 32, 0, c->stream>>>(partial, c->d_tensor_chunk_begin, out, nt);
     c->launches++;
     CU(c, cudaGetLastError());
@@ -369,6 +370,7 @@ int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int*
     }
     if (c->cfg.flags & HALOS_FLAG_STATS) {
         if ((rc = finalize_stats(c, 0, lps)) != HALOS_OK) return rc;
+        if ((rc = finalize_stats(c, 2, lps)) != HALOS_OK) return rc;
         if (push && (rc = finalize_stats(c, 1, lps)) != HALOS_OK) return rc;
     }
     apply_commit(c, lps, worker, push);
@@ -545,7 +547,8 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     if (cfg->flags & HALOS_FLAG_STATS) {
         ok &= (c->d_partial_delta = (double*)A(nc * 8)) != nullptr;
         ok &= (c->d_partial_Delta = (double*)A(nc * 8)) != nullptr;
-        ok &= (c->d_stats = (double*)A((size_t)2 * cfg->n_lps * nt * 8)) != nullptr;
+        ok &= (c->d_partial_theta = (double*)A(nc * 8)) != nullptr;
+        ok &= (c->d_stats = (double*)A((size_t)3 * cfg->n_lps * nt * 8)) != nullptr;
     }
     ok &= (c->Theta = (float*)S(P * 4)) != nullptr;
     ok &= (c->Mg = (float*)S(P * 4)) != nullptr;
@@ -587,7 +590,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     CUC(cudaMemcpyAsync(c->d_chunks, c->chunks.data(), nc * sizeof(Chunk), cudaMemcpyHostToDevice, st));
     CUC(cudaMemcpyAsync(c->d_tensor_off, c->tensor_off.data(), (nt + 1) * 8, cudaMemcpyHostToDevice, st));
     CUC(cudaMemcpyAsync(c->d_tensor_chunk_begin, c->tensor_chunk_begin.data(), (nt + 1) * 4, cudaMemcpyHostToDevice, st));
-    if (c->d_stats) CUC(cudaMemsetAsync(c->d_stats, 0, (size_t)2 * cfg->n_lps * nt * 8, st));
+    if (c->d_stats) CUC(cudaMemsetAsync(c->d_stats, 0, (size_t)3 * cfg->n_lps * nt * 8, st));
     // Alg. 1 lines 6-7
     CUC(cudaMemcpyAsync(c->Theta, theta_init_dev, P * 4, cudaMemcpyDeviceToDevice, st));
     CUC(cudaMemsetAsync(c->Mg, 0, P * 4, st));
@@ -1054,7 +1057,7 @@ int halos_worker_info(halos_ctx* c, uint32_t worker, uint64_t* out) {
 int halos_stats(halos_ctx* c, uint32_t what, uint32_t lps, double* out) {
     if (!c || !out) return HALOS_ERR_INVALID_ARG;
     if (!(c->cfg.flags & HALOS_FLAG_STATS)) return fail(c, HALOS_ERR_BAD_STATE, "context was created without HALOS_FLAG_STATS");
-    if (what > 1 || lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "bad statistic or lps");
+    if (what > 2 || lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "bad statistic or lps");
     const size_t nt = c->tensor_numel.size();
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaMemcpyAsync(out, c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt, nt * 8, cudaMemcpyDeviceToHost, c->stream));

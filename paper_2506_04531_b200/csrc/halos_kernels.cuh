@@ -240,6 +240,7 @@ struct ArriveArgs {
     float* outbox;              // Delta               (PUSH only)
     double* partial_delta;      // [n_chunks] sum delta^2 per chunk (STATS only)
     double* partial_Delta;      // [n_chunks] sum Delta^2 per chunk (STATS && PUSH)
+    double* partial_theta;      // [n_chunks] sum theta_t^2 of the updated LPS model per chunk (STATS only)
     float eta, beta, omb;
 };
 
@@ -262,7 +263,7 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
     const float* an = PUSH ? a.anchor + c.begin : nullptr;
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eta = a.eta, beta = a.beta, omb = a.omb;
-    float acc_d = 0.f, acc_D = 0.f;
+    float acc_d = 0.f, acc_D = 0.f, acc_x = 0.f;
 
     // vector path: the chunk starts on a VE-element boundary of the packed state (bases are 256-byte
     // aligned) and the caller's theta_H pointer is aligned to one vector of its own type
@@ -298,7 +299,10 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
                     stf<VE, STREAM>(th + o, vx[u]);
                     stf<VE, STREAM>(ml + o, vm[u]);
                     T::template store<VE, STREAM>(s0 + o, vx[u]);
-                    if (STATS) acc_d = sumsq<VE>(d, acc_d);
+                    if (STATS) {
+                        acc_d = sumsq<VE>(d, acc_d);
+                        acc_x = sumsq<VE>(vx[u], acc_x);
+                    }
                     if (PUSH) {
                         FVec<VE> D;
 #pragma unroll
@@ -319,7 +323,10 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
         th[j] = x;
         ml[j] = m;
         T::store1(s0 + j, x);
-        if (STATS) acc_d = fmaf(d, d, acc_d);
+        if (STATS) {
+            acc_d = fmaf(d, d, acc_d);
+            acc_x = fmaf(x, x, acc_x);
+        }
         if (PUSH) {
             float D = __fsub_rn(x, an[j]);
             ob[j] = D;
@@ -330,6 +337,9 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
         __shared__ double red[kThreads / 32];
         double t = block_sum((double)acc_d, red);
         if (threadIdx.x == 0) a.partial_delta[blockIdx.x] = t;
+        __syncthreads();
+        double t3 = block_sum((double)acc_x, red);
+        if (threadIdx.x == 0) a.partial_theta[blockIdx.x] = t3;
         if (PUSH) {
             __syncthreads();
             double t2 = block_sum((double)acc_D, red);

@@ -283,6 +283,7 @@ def test_norm_statistics():
         rec = ls.step(ev)
         if rec["kind"] == tr.ARRIVE:
             np.testing.assert_allclose(ls.h.stats(0, rec["lps"]), ls.o.sq_norms("delta", rec["lps"], off), rtol=2e-6)
+            np.testing.assert_allclose(ls.h.stats(2, rec["lps"]), ls.o.sq_norms("th", rec["lps"], off), rtol=2e-6)
             if rec["pushed"]:
                 np.testing.assert_allclose(ls.h.stats(1, rec["lps"]), ls.o.sq_norms("outbox", rec["lps"], off), rtol=2e-6)
     ls.compare(ls.all_buffers(), FULL_TRACE_TOL)
@@ -644,3 +645,84 @@ def test_materialised_delta_frees_the_callers_buffer():
     with pytest.raises(hb.HalosError) as e:
         hb.Halos(torch.zeros(8, device="cuda"), [0], flags=hb.FLAG_MATERIALISE_DELTA | hb.FLAG_STATS)
     assert e.value.status == hb.ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------------------------------------
+# random call sequences, legal and illegal, against a reference state machine and the oracle
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(3))
+def test_api_fuzz_statuses_and_state(seed):
+    from oracle import HalosOracle
+    rng = np.random.default_rng(500 + seed)
+    lay = layouts.ragged_layout("f", [129, 7, 64, 1, 300])
+    worker_lps = [0, 0, 1, 2, 2]
+    n_lps, K = 3, 10 ** 6                       # pushes happen when the fuzzer says so, not on a window
+    init = gen.theta_init(lay, 70 + seed)
+    h = hb.Halos(torch.from_numpy(init).cuda(), worker_lps, lay.numel, K=K, flags=hb.FLAG_GUARD, **PAPER_HP)
+    o = HalosOracle(init, worker_lps, K=K, **PAPER_HP)
+    pending = {}                                # worker -> result (numpy) registered but not applied
+    keep = {}
+    phase = [hb.IDLE] * n_lps
+    n_ok = n_bad = 0
+    for step in range(700):
+        op = int(rng.integers(0, 5))
+        l, w = int(rng.integers(0, n_lps + 1)), int(rng.integers(0, len(worker_lps) + 1))   # sometimes out of range
+        if rng.random() < 0.85:                 # mostly well-formed arguments, so that the state really advances
+            l, w = min(l, n_lps - 1), min(w, 4)
+            if op == 1 and rng.random() < 0.8:
+                l = worker_lps[w]
+        want, call = hb.OK, None
+        if op == 0:
+            res = gen.worker_result(o.buffer("th0", min(w, 4)), lay, 70 + seed, min(w, 4), step)
+            cand = torch.from_numpy(res).cuda()
+            call = lambda: h.worker_delta(w, cand)
+            want = hb.ERR_INVALID_ARG if w >= 5 else (hb.ERR_BAD_STATE if w in pending else hb.OK)
+            if want == hb.OK:
+                pending[w] = res
+                keep[w] = cand                  # borrowed by the library until the apply: keep it alive
+        elif op == 1:
+            call = lambda: h.lps_apply(l, w)
+            if l >= n_lps or w >= 5 or worker_lps[w] != l:
+                want = hb.ERR_INVALID_ARG
+            elif w not in pending:
+                want = hb.ERR_BAD_STATE
+            else:
+                o.arrive(w, pending.pop(w))
+        elif op == 2:
+            call = lambda: h.lps_push(l)
+            want = hb.ERR_INVALID_ARG if l >= n_lps else (hb.ERR_BAD_STATE if phase[l] != hb.IDLE else hb.OK)
+            if want == hb.OK:
+                o.push(l)
+                phase[l] = hb.PUSHED
+        elif op == 3:
+            call = lambda: h.gps_merge(l)
+            want = hb.ERR_INVALID_ARG if l >= n_lps else (hb.ERR_BAD_STATE if phase[l] != hb.PUSHED else hb.OK)
+            if want == hb.OK:
+                o.gps_recv(l)
+                phase[l] = hb.ANSWERED
+        else:
+            call = lambda: h.lps_pull(l)
+            want = hb.ERR_INVALID_ARG if l >= n_lps else (hb.ERR_BAD_STATE if phase[l] != hb.ANSWERED else hb.OK)
+            if want == hb.OK:
+                o.pull(l)
+                phase[l] = hb.IDLE
+        if want == hb.OK:
+            call()
+            n_ok += 1
+        else:
+            with pytest.raises(hb.HalosError) as e:
+                call()
+            assert e.value.status == want, (step, op, l, w)
+            n_bad += 1
+    assert n_ok > 150 and n_bad > 150
+    for l in range(n_lps):
+        assert h.counters(l) == o.counters(l)
+        for which, name in ((hb.BUF_THETA_L, "th"), (hb.BUF_M_L, "ml"), (hb.BUF_ANCHOR, "anchor"),
+                            (hb.BUF_OUTBOX, "outbox"), (hb.BUF_INBOX, "inbox")):
+            assert np.array_equal(h.read(which, l).view(np.uint32), o.buffer(name, l).view(np.uint32)), (name, l)
+    assert np.array_equal(h.read(hb.BUF_THETA_G).view(np.uint32), o.buffer("Theta").view(np.uint32))
+    assert np.array_equal(h.read(hb.BUF_M_G).view(np.uint32), o.buffer("Mg").view(np.uint32))
+    for w in range(5):
+        assert np.array_equal(h.read(hb.BUF_THETA0, w).view(np.uint32), o.buffer("th0", w).view(np.uint32))
+    assert h.check_guards() == -1
+    h.close()
