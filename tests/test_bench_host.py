@@ -57,3 +57,60 @@ def test_reference_arm_line():
     line = json.loads(out)
     assert line["impl"] == "reference" and line["metric"] == "params_updated_per_sec" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def _shard_main(rank, world, port, out_dir):
+    """Index-sharded replicas: every rank replays the same trace on its own contiguous slice of the
+    parameter vector; no exchange is needed on the data path (the method is elementwise)."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, str(ROOT))
+    from oracle import HalosOracle
+    from paper_2506_04531_b200.inputs import gen, layouts, trace as tr
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    lay = layouts.ragged_layout("s", [1000, 37, 4096, 3, 2000])
+    P = lay.P
+    lo, hi = rank * P // world, (rank + 1) * P // world
+    worker_lps = [0, 0, 1, 1]
+    events = tr.random_trace(worker_lps, 80, 3, seed=4)
+    o = HalosOracle(gen.theta_init(lay, 5, lo, hi), worker_lps, K=3)
+    for ev in events:
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        if kind == tr.ARRIVE:
+            o.arrive(w, gen.worker_result(o.buffer("th0", w), lay, 5, w, o.worker_info(w)["round"], lo, hi))
+        elif kind == tr.GPS_RECV:
+            o.gps_recv(l)
+        else:
+            o.pull(l)
+    mine = torch.from_numpy(np.concatenate([o.buffer("Theta"), o.buffer("th", 1)]).copy())
+    assert P % world == 0                      # equal shards, so a plain all_gather collects the result
+    parts = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(parts, mine)               # only to collect the answer; the replay itself exchanged nothing
+    if rank == 0:
+        np.save(Path(out_dir, "gathered.npy"), np.concatenate([p.numpy() for p in parts]))
+    dist.destroy_process_group()
+
+
+def test_index_sharded_replicas_gloo(tmp_path):
+    import torch.multiprocessing as mp
+    from oracle import HalosOracle
+    from paper_2506_04531_b200.inputs import gen, layouts, trace as tr
+    port = 31500 + (os.getpid() % 2000)
+    mp.spawn(_shard_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    got = np.load(tmp_path / "gathered.npy")
+    lay = layouts.ragged_layout("s", [1000, 37, 4096, 3, 2000])
+    P = lay.P
+    worker_lps = [0, 0, 1, 1]
+    o = HalosOracle(gen.theta_init(lay, 5), worker_lps, K=3)
+    for ev in tr.random_trace(worker_lps, 80, 3, seed=4):
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        if kind == tr.ARRIVE:
+            o.arrive(w, gen.worker_result(o.buffer("th0", w), lay, 5, w, o.worker_info(w)["round"]))
+        elif kind == tr.GPS_RECV:
+            o.gps_recv(l)
+        else:
+            o.pull(l)
+    half = P // 2
+    want = np.concatenate([o.buffer("Theta")[:half], o.buffer("th", 1)[:half], o.buffer("Theta")[half:], o.buffer("th", 1)[half:]])
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
