@@ -726,3 +726,43 @@ def test_api_fuzz_statuses_and_state(seed):
         assert np.array_equal(h.read(hb.BUF_THETA0, w).view(np.uint32), o.buffer("th0", w).view(np.uint32))
     assert h.check_guards() == -1
     h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# plumbing variants: a non-default stream, the library's own cudaMalloc, two contexts interleaved
+# ---------------------------------------------------------------------------------------------
+def test_side_stream_own_allocator_and_interleaved_contexts():
+    from oracle import HalosOracle
+    lay = layouts.ragged_layout("p", [5000, 3, 12345, 64])
+    init = gen.theta_init(lay, 41)
+    worker_lps = [0, 1, 1]
+    side = torch.cuda.Stream()
+    init_dev = torch.from_numpy(init).cuda()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        a = hb.Halos(init_dev, worker_lps, lay.numel, K=2, stream=side, **PAPER_HP)
+    b = hb.Halos(init_dev, worker_lps, lay.numel, K=2, use_torch_allocator=False, **PAPER_HP)
+    oa = HalosOracle(init, worker_lps, K=2, **PAPER_HP)
+    events = tr.random_trace(worker_lps, 60, 2, seed=3)
+    keep = []
+    for ev in events:
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        if kind == tr.ARRIVE:
+            res = gen.worker_result(oa.buffer("th0", w), lay, 41, w, oa.worker_info(w)["round"])
+            t = torch.from_numpy(res).cuda()
+            torch.cuda.synchronize()               # the input is complete before either stream reads it
+            keep.append(t)
+            for h in (a, b):                       # the two contexts take turns, each on its own stream
+                h.worker_delta(w, t)
+                if h.lps_apply(l, w):
+                    h.lps_push(l)
+            oa.arrive(w, res)
+        elif kind == tr.GPS_RECV:
+            a.gps_merge(l); b.gps_merge(l); oa.gps_recv(l)
+        else:
+            a.lps_pull(l); b.lps_pull(l); oa.pull(l)
+    for h in (a, b):
+        for l in (0, 1):
+            assert np.array_equal(h.read(hb.BUF_THETA_L, l).view(np.uint32), oa.buffer("th", l).view(np.uint32))
+        assert np.array_equal(h.read(hb.BUF_THETA_G).view(np.uint32), oa.buffer("Theta").view(np.uint32))
+        h.close()
