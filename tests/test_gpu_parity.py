@@ -766,3 +766,65 @@ def test_side_stream_own_allocator_and_interleaved_contexts():
             assert np.array_equal(h.read(hb.BUF_THETA_L, l).view(np.uint32), oa.buffer("th", l).view(np.uint32))
         assert np.array_equal(h.read(hb.BUF_THETA_G).view(np.uint32), oa.buffer("Theta").view(np.uint32))
         h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# configuration 2 (70M, bf16 copies): EVERY element of every buffer after 500 events.  The oracle runs
+# one independent replayer per core on a contiguous slice (elementwise method), fed by the C generator.
+# ---------------------------------------------------------------------------------------------
+def test_config_70m_every_element():
+    import concurrent.futures as cf
+    import os
+    from oracle import HalosOracle
+    from paper_2506_04531_b200.inputs.gen_c import HostGenerator
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    wl = workloads.workload("70m")
+    lay, P = wl.layout, wl.layout.P
+    events = wl.trace()[:500]
+    assert int((events["kind"] == tr.PULL).sum()) >= 8
+
+    # CUDA side: full size, batched driver, per-worker result buffers
+    dg = DeviceGenerator(lay, wl.seed)
+    h = hb.Halos(dg.theta_init(), wl.worker_lps, lay.numel, worker_dtype=wl.worker_dtype, **wl.hyper())
+    bufs = [torch.empty(P, dtype=torch.int16, device="cuda") for _ in range(wl.n_workers)]
+
+    def producer(index, worker, rnd):
+        return dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker], worker_dtype=wl.worker_dtype)
+
+    h.replay(events, producer, max_batch=8)
+    names = [("Theta", hb.BUF_THETA_G, 0), ("Mg", hb.BUF_M_G, 0)]
+    for l in range(wl.n_lps):
+        names += [(n, b, l) for n, b in (("th", hb.BUF_THETA_L), ("ml", hb.BUF_M_L), ("anchor", hb.BUF_ANCHOR),
+                                         ("outbox", hb.BUF_OUTBOX), ("inbox", hb.BUF_INBOX))]
+    names += [("th0", hb.BUF_THETA0, w) for w in range(wl.n_workers)]
+    gpu = {(n, i): h.read(b, i) for n, b, i in names}
+    h.close()
+    del bufs
+    torch.cuda.empty_cache()
+
+    # oracle side: slices in parallel threads (the C calls release the GIL)
+    cores = max(1, min(16, len(os.sched_getaffinity(0))))
+    cuts = [P * k // cores for k in range(cores + 1)]
+    hg = HostGenerator(lay, wl.seed)
+
+    def run_slice(k):
+        lo, hi = cuts[k], cuts[k + 1]
+        o = HalosOracle(hg.theta_init(lo, hi), wl.worker_lps, worker_dtype=wl.worker_dtype, **wl.hyper())
+        for ev in events:
+            kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+            if kind == tr.ARRIVE:
+                o.arrive(w, hg.worker_result(o.buffer("th0", w), w, o.worker_info(w)["round"], lo, wl.worker_dtype))
+            elif kind == tr.GPS_RECV:
+                o.gps_recv(l)
+            else:
+                o.pull(l)
+        bad = []
+        for n, _, i in names:
+            if not np.array_equal(gpu[(n, i)][lo:hi].view(np.uint16), o.buffer(n, i).view(np.uint16)):
+                bad.append((n, i, lo))
+        o.close()
+        return bad
+
+    with cf.ThreadPoolExecutor(max_workers=cores) as ex:
+        bad = [b for part in ex.map(run_slice, range(cores)) for b in part]
+    assert not bad, bad[:5]

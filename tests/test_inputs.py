@@ -154,3 +154,18 @@ def test_paper_cluster_options():
     hg = workloads.workload("hetero_grouping_small")
     assert hg.n_lps == 8 and sorted(set(hg.worker_lps)) == list(range(8))
     assert hg.lps_gbps[5] == hg.lps_gbps[7] == 0.202 and hg.lps_gbps[0] == 100.0
+
+
+def test_c_generator_equals_numpy_generator():
+    from paper_2506_04531_b200.inputs.gen_c import HostGenerator
+    for lay in (layouts.decoder_layout("tiny", 2, 64, 300), layouts.ragged_layout("e", [16, 0, 5, 0, 64, 1, 4099])):
+        hg = HostGenerator(lay, 77)
+        init = gen.theta_init(lay, 77)
+        np.testing.assert_array_equal(hg.theta_init().view(np.uint32), init.view(np.uint32))
+        lo, hi = 17, lay.P - 9
+        np.testing.assert_array_equal(hg.theta_init(lo, hi), init[lo:hi])
+        np.testing.assert_array_equal(hg.worker_result(init[lo:hi], 3, 9, lo).view(np.uint32),
+                                      gen.worker_result(init[lo:hi], lay, 77, 3, 9, lo, hi).view(np.uint32))
+        hb16 = gen.f32_to_bf16_bits(init)
+        np.testing.assert_array_equal(hg.worker_result(hb16[lo:hi], 3, 9, lo, gen.BF16),
+                                      gen.worker_result(hb16[lo:hi], lay, 77, 3, 9, lo, hi, gen.BF16))
