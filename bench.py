@@ -161,8 +161,10 @@ class OracleReplayer:
         from oracle import HalosOracle
         from paper_2506_04531_b200.inputs import gen
         self.wl, self.lay = wl, wl.layout
+        from paper_2506_04531_b200.inputs.gen_c import HostGenerator
         self.S = min(slice_params, self.lay.P)
-        init = gen.theta_init(self.lay, wl.seed, 0, self.S)
+        self.hg = HostGenerator(self.lay, wl.seed)
+        init = self.hg.theta_init(0, self.S)
         self.o = HalosOracle(init, wl.worker_lps, worker_dtype=wl.worker_dtype, dtype=np.float32, **wl.hyper())
 
     def run(self, events, budget_s: float = float("inf")):
@@ -174,7 +176,7 @@ class OracleReplayer:
             kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
             if kind == tr.ARRIVE:
                 r = o.worker_info(w)["round"]
-                thH = gen.worker_result(o.buffer("th0", w), self.lay, wl.seed, w, r, 0, self.S, wl.worker_dtype)   # untimed input
+                thH = self.hg.worker_result(o.buffer("th0", w), w, r, 0, wl.worker_dtype)   # untimed input
                 t0 = time.perf_counter()
                 o.arrive(w, thH)
             elif kind == tr.GPS_RECV:
@@ -337,7 +339,7 @@ def main():
         events = window_events(args.steps + args.warmup, args.events_per_step, wl)
         # every step replays its whole window (the state carries over), on an index slice small enough
         # for the run to end within a few minutes
-        S = min(1 << 20, P)
+        S = min(1 << 22, P)
         rep = OracleReplayer(wl, S)
         t_total, total_done = 0.0, 0
         for s in range(args.steps + args.warmup):
