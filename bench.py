@@ -499,6 +499,9 @@ def main():
         main_run = timed_region(args.max_batch, n_steps)  # multi-event fusion in the driver
     else:
         main_run = per_event
+    for which, idx in [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]:
+        if not np.isfinite(h.read(which, idx, 0, 4096)).all():
+            raise SystemExit("non-finite model values after the timed region")
     value, roofline, launches = main_run["value"], main_run["roofline"], main_run["launches"]
     t_ms = main_run["ms_per_step"] * args.steps
 
