@@ -17,10 +17,13 @@
  *  - All state buffers are flat, packed in tensor order (tensor k starts at the sum of the
  *    sizes before it), fp32 except worker snapshots (worker_dtype).  The context OWNS them.
  *  - Pointers named *_dev are device pointers on the context's device, *_host are host pointers.
- *  - All device work is enqueued on the stream given at creation; calls are asynchronous and
- *    stream ordered.  Host-side counters (t, t_last, i, phases) change at enqueue time.
- *  - Every call returns a status; on any status other than HALOS_OK the context's state is
- *    unchanged and out-parameters are not written.  Nothing aborts or traps.
+ *  - All kernels are enqueued on the stream given at creation; calls are asynchronous and stream
+ *    ordered.  (Only the host-to-device copies of halos_worker_delta_host run on a second stream
+ *    that the context owns; events tie them to the kernels that read them.)  Host-side counters
+ *    (t, t_last, i, phases) change at enqueue time.
+ *  - Status HALOS_ERR_CUDA means the CUDA runtime reported an error: treat the context as lost.
+ *  - Every call returns a status; on any other status than HALOS_OK (HALOS_ERR_CUDA excepted) the
+ *    context's state is unchanged and out-parameters are not written.  Nothing aborts or traps.
  *  - A context is not thread safe.  There is no CPU fallback: without a CUDA device
  *    halos_create fails with HALOS_ERR_CUDA.
  */
@@ -132,8 +135,12 @@ int halos_worker_delta(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_
                        const void* const* thetaH_ptrs_host);
 
 /* Same, for a result that sits in HOST memory (P elements of worker_dtype, packed): it is copied
- * into a context-owned staging buffer on the stream (pinned host memory makes the copy
- * asynchronous), so the borrow ends when that copy has completed in stream order. */
+ * into one of two context-owned staging buffers (allocated on first use) by a copy stream the
+ * context owns, ordered against the update kernels with events, so that the copy of the next result
+ * overlaps the kernel of the current one; pinned host memory makes the copy asynchronous.  The host
+ * data is borrowed until that copy has completed.  BAD_STATE if both staging buffers still hold
+ * results that were not applied (at most two host results may be pending), OOM if a staging buffer
+ * cannot be allocated. */
 int halos_worker_delta_host(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_host);
 
 /* Alg. 1 lines 10-13 at LPS `lps` for the pending result of `worker`:  t <- t+1;
