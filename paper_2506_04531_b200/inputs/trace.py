@@ -150,3 +150,16 @@ def random_trace(n_workers_lps: Sequence[int], n_events: int, K: int, seed: int)
             phase[l] = 0
             t_last[l] = t[l]
     return np.array(events, dtype=EVENT_DTYPE)
+
+
+def save_trace(path, events: np.ndarray) -> None:
+    """Trace file = the flat little-endian array of 16-byte records {u8 kind, u8 lps, u16 worker, u32 pad,
+    i64 time_ns}; the same layout the C driver takes."""
+    np.ascontiguousarray(events, dtype=EVENT_DTYPE).tofile(str(path))
+
+
+def load_trace(path) -> np.ndarray:
+    ev = np.fromfile(str(path), dtype=EVENT_DTYPE)
+    if ev.size and int(ev["kind"].max()) > PULL:
+        raise ValueError("not a trace file: unknown event kind")
+    return ev

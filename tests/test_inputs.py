@@ -169,3 +169,13 @@ def test_c_generator_equals_numpy_generator():
         hb16 = gen.f32_to_bf16_bits(init)
         np.testing.assert_array_equal(hg.worker_result(hb16[lo:hi], 3, 9, lo, gen.BF16),
                                       gen.worker_result(hb16[lo:hi], lay, 77, 3, 9, lo, hi, gen.BF16))
+
+
+def test_trace_file_round_trip(tmp_path):
+    ev = workloads.workload("toy_k4").trace()
+    tr.save_trace(tmp_path / "toy.trace", ev)
+    assert (tmp_path / "toy.trace").stat().st_size == 16 * len(ev)
+    np.testing.assert_array_equal(tr.load_trace(tmp_path / "toy.trace"), ev)
+    (tmp_path / "junk").write_bytes(bytes(range(32)))
+    with pytest.raises(ValueError):
+        tr.load_trace(tmp_path / "junk")
