@@ -533,6 +533,7 @@ def main():
         e2e = {"value": u_all / (dt_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": int(arrivals / e2e_steps * P * (4 if wl.worker_dtype == gen.F32 else 2)),
                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps}
+        e2e["h2d_GBps"] = e2e["h2d_bytes_per_step"] / (e2e["ms_per_step"] * 1e6)   # the PCIe copy bounds this leg
         del host_results
 
     h.close()

@@ -21,6 +21,8 @@
  *    ordered.  (Only the host-to-device copies of halos_worker_delta_host run on a second stream
  *    that the context owns; events tie them to the kernels that read them.)  Host-side counters
  *    (t, t_last, i, phases) change at enqueue time.
+ *  - Calls that touch the device make the context's device the calling thread's current CUDA device
+ *    and leave it so.
  *  - Status HALOS_ERR_CUDA means the CUDA runtime reported an error: treat the context as lost.
  *  - Every call returns a status; on any other status than HALOS_OK (HALOS_ERR_CUDA excepted) the
  *    context's state is unchanged and out-parameters are not written.  Nothing aborts or traps.
