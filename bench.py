@@ -5,10 +5,13 @@
 
 A step replays the next ``--events-per-step`` events (worker arrivals with their pushes, GPS
 updates, merges) of the workload's seeded asynchronous trace through the library's event-queue
-driver: one fused kernel per event over all tensors of the model.  Metric: parameters updated per
-second (every event updates the P parameters of one model).
+driver.  Metric: parameters updated per second (every event updates the P parameters of one model).
+Worker results are the faithful theta_H = theta_0 + noise of every arrival: the timed steps are run
+once untimed with the generator in the loop, each result is kept in HBM, the state is rebuilt and
+the timed runs read the resident results (and must end in the same state, which is checked).  The
+step length is reduced from 128 events until the results of all timed steps fit in device memory.
 
-    value       device-resident: each worker's result theta_H already sits in HBM; the driver fuses up to
+    value       device-resident: every arrival's result theta_H already sits in HBM; the driver fuses up to
                 --max-batch arrivals at one LPS into one launch (bit-identical to one launch per
                 event, which is measured too and reported under per_event_kernels)
     e2e         the same replay through the C ABI with HOST-resident worker results (pinned), the
@@ -302,7 +305,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "410m", "70m_f32_small"])
-    ap.add_argument("--events-per-step", type=int, default=128)
+    ap.add_argument("--events-per-step", type=int, default=0,
+                    help="events per step; 0 = 128, reduced so that the results of all timed steps fit in HBM")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
@@ -328,7 +332,7 @@ def main():
     wname = {0: "f32", 1: "bf16"}[wl.worker_dtype]
     config = {"workload": f"{wl.name}: decoder layout P={P} ({lay.n_tensors} tensors), {wl.n_workers} workers over "
                           f"{wl.n_lps} LPS, 1 GPS, fp32 master + {wname} worker copies, K={wl.K}, paper hyperparameters",
-              "events_per_step": args.events_per_step, "trace_seed": wl.seed, "max_batch": args.max_batch,
+              "events_per_step": args.events_per_step or 128, "trace_seed": wl.seed, "max_batch": args.max_batch,
               "l2": "every buffer (%.0f MB) is larger than L2; no flush needed" % (P * 4 / 1e6),
               "parallelism": "index-sharded replicas, no collective" if world > 1 else "single GPU"}
 
@@ -336,14 +340,15 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        events = window_events(args.steps + args.warmup, args.events_per_step, wl)
+        eps_ref = args.events_per_step or 128
+        events = window_events(args.steps + args.warmup, eps_ref, wl)
         # every step replays its whole window (the state carries over), on an index slice small enough
         # for the run to end within a few minutes
         S = min(1 << 22, P)
         rep = OracleReplayer(wl, S)
         t_total, total_done = 0.0, 0
         for s in range(args.steps + args.warmup):
-            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
+            win = events[s * eps_ref:(s + 1) * eps_ref]
             spent, done = rep.run(win)
             if s >= args.warmup:
                 t_total += spent
@@ -355,7 +360,7 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic", "config": config,
                 "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                 "sample": f"every step's {args.events_per_step} events on the index slice [0,{S}) of {P} parameters"},
+                                 "sample": f"every step's {eps_ref} events on the index slice [0,{S}) of {P} parameters"},
                 "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "gpu_launches": 0}
         print(json.dumps(line))
@@ -379,74 +384,81 @@ def main():
     from paper_2506_04531_b200.inputs import gen
     from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
 
-    n_steps = args.steps + args.warmup
-    events = window_events(n_steps * 2 + 8, args.events_per_step, wl)
+    # ------------------------------------------------------------------ inputs of the timed regions
+    # A worker's result is theta_H = theta_0 + noise, where theta_0 is the model the LPS last scheduled
+    # it: it depends on the state.  (Feeding fixed targets instead turns the asynchronous hierarchy into
+    # an unstable control loop and the models overflow within a few thousand events.)  To time with the
+    # true values AND with every input resident in HBM, the K timed steps are first executed once,
+    # untimed, with the generator in the loop, and every result is kept in its own buffer; the state is
+    # then rebuilt (same seed, same warm-up: bit-identical) and the timed runs read the stored results.
+    # The number of results that fit in HBM bounds the length of a step.
+    wbytes = 4 if wl.worker_dtype == gen.F32 else 2
+    wdt = torch.float32 if wl.worker_dtype == gen.F32 else torch.int16
+    n_state_bufs = 2 + 5 * wl.n_lps
+    state_bytes = n_state_bufs * 4 * P + wl.n_workers * wbytes * P
+    free_b, total_b = torch.cuda.mem_get_info(dev)
+    room = int(0.88 * (free_b - state_bytes - 3 * wbytes * P - (2 << 30)))
+    fit_arrivals = max(1, room // (wbytes * P))
+    eps = args.events_per_step if args.events_per_step > 0 else 128
+    eps = int(max(1, min(eps, (fit_arrivals * 100 // 96) // max(1, args.steps))))   # ~96% of the events are arrivals
+    K, W = args.steps, args.warmup
+    events = window_events(W + K, eps, wl)
+    from paper_2506_04531_b200.inputs import trace as tr
+    timed_events = events[W * eps:(W + K) * eps]
+    arrive_slots = {int(i): n for n, i in enumerate(np.nonzero(timed_events["kind"] == tr.ARRIVE)[0])}
+    n_timed_arrivals = len(arrive_slots)
+    if n_timed_arrivals > fit_arrivals:
+        raise SystemExit(f"{n_timed_arrivals} resident results do not fit in device memory (room for {fit_arrivals})")
+    config["events_per_step"] = eps
+    config["inputs"] = (f"theta_H = theta_0 + sigma z per arrival (faithful), {n_timed_arrivals} results of the timed steps "
+                        f"pre-generated by an untimed pass and resident in HBM ({n_timed_arrivals * wbytes * P / 1e9:.1f} GB)")
+
     seed = wl.seed + 1000 * rank                      # each rank: its own shard of a larger model
     dgen = DeviceGenerator(lay, seed, device=dev)
-    init = dgen.theta_init()
-    h = hb.Halos(init, wl.worker_lps, lay.numel, worker_dtype=wl.worker_dtype, chunk_elems=args.chunk_elems, **wl.hyper())
-    wdt = torch.float32 if wl.worker_dtype == gen.F32 else torch.int16
-    # device-resident worker results: one buffer per worker, theta_H = Theta_0 + sigma z_w
-    results = [dgen.worker_result(h.peek(hb.BUF_THETA0, w), w, 0, worker_dtype=wl.worker_dtype)
-               for w in range(wl.n_workers)]
-    del init
-    torch.cuda.synchronize(dev)
+    scratch = torch.empty(P, dtype=wdt, device=dev)   # warm-up results (one at a time: max_batch = 1)
 
-    def producer_dev(index, worker, rnd):
-        return results[worker]
+    def fresh_context():
+        """A context in the state right before the first timed step (deterministic)."""
+        init = dgen.theta_init()
+        h = hb.Halos(init, wl.worker_lps, lay.numel, worker_dtype=wl.worker_dtype, chunk_elems=args.chunk_elems, **wl.hyper())
+        del init
 
-    def run_step(s, e2e=False, host_results=None, probe=None):
-        win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
-        # end to end: results live in pinned host memory and are copied in by the library; two
-        # staging buffers let the copy of the next result overlap the current update kernel
-        from paper_2506_04531_b200.inputs import trace as tr
-        pend = []
-        n = len(win)
-        nxt = 0
+        def gen_into_scratch(index, worker, rnd):
+            return dgen.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=scratch, worker_dtype=wl.worker_dtype)
+        for s in range(W):
+            h.replay(events[s * eps:(s + 1) * eps], gen_into_scratch, want_log=False, max_batch=1)
+        return h
 
-        def feed():
-            nonlocal nxt
-            while nxt < n and len(pend) < 2:
-                ev = win[nxt]
-                if int(ev["kind"]) == tr.ARRIVE:
-                    w = int(ev["worker"])
-                    if any(int(win[p]["worker"]) == w for p in pend):
-                        break
-                    h.worker_delta_host(w, host_results[w])
-                    pend.append(nxt)
-                nxt += 1
-        for k in range(n):
-            nxt = max(nxt, k)
-            feed()
-            ev = win[k]
-            kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
-            if kind == tr.ARRIVE:
-                assert pend and pend[0] == k
-                pend.pop(0)
-                if h.lps_apply(l, w):
-                    h.lps_push(l)
-                feed()
-            elif kind == tr.GPS_RECV:
-                h.gps_merge(l)
-            else:
-                h.lps_pull(l)
-        # device -> host read of the step's result: a probe of the global and local models
-        got = 0
-        for which, idx in probe:
-            got += h.read(which, idx, 0, 1024).nbytes
-        return got
+    def state_digest(h):
+        """Order-independent 64-bit checksums of the models (to check that the runs ended in the same state)."""
+        out = []
+        for which, idx in [(hb.BUF_THETA_G, 0), (hb.BUF_M_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]:
+            t = h.peek(which, idx)
+            if not bool(torch.isfinite(t).all()):
+                raise SystemExit("non-finite model values")
+            out.append(int(t.view(torch.int32).to(torch.int64).sum().item()))
+        return out
 
-    # ---- warm-up, then the timed region (device-resident); once per driver mode ----
+    # ---- untimed pass: generate and keep the results of the K timed steps ----
+    resident = torch.empty((n_timed_arrivals, P), dtype=wdt, device=dev)
+    h = fresh_context()
+    for s in range(K):
+        base = s * eps
+
+        def gen_and_keep(index, worker, rnd, base=base):
+            return dgen.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=resident[arrive_slots[base + index]],
+                                      worker_dtype=wl.worker_dtype)
+        h.replay(timed_events[base:base + eps], gen_and_keep, want_log=False, max_batch=1)
+    want_digest = state_digest(h)
+    h.close()
+    del h
+    torch.cuda.empty_cache()
+
     peak, peak_kind = measured_peak_gbs()
-    wbytes = 4 if wl.worker_dtype == gen.F32 else 2
 
-    def timed_region(max_batch, first_step):
-        """W warm-up + K timed steps starting at window `first_step`; returns the measurements."""
-        def step(s):
-            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
-            h.replay(win, producer_dev, want_log=False, max_batch=max_batch)
-        for s in range(first_step, first_step + args.warmup):
-            step(s)
+    def timed_region(max_batch):
+        """K timed steps from the state after the warm-up, reading the resident results."""
+        h = fresh_context()
         torch.cuda.synchronize(dev)
         h.timing_enable(True)
         launches0, batch0 = h.info()["launches"], h.batch_info()
@@ -454,10 +466,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with ClockSampler(local_rank) as clk:
+        with ClockSampler(local_rank, period_s=0.01) as clk:
             e0.record()
-            for s in range(first_step + args.warmup, first_step + n_steps):
-                step(s)
+            for s in range(K):
+                base = s * eps
+                h.replay(timed_events[base:base + eps], lambda index, worker, rnd, base=base: resident[arrive_slots[base + index]],
+                         want_log=False, max_batch=max_batch)
             e1.record()
             torch.cuda.synchronize(dev)
         if world > 1:
@@ -466,7 +480,10 @@ def main():
         launches = h.info()["launches"] - launches0
         timing, batch1 = h.timing_read(), h.batch_info()
         h.timing_enable(False)
-        units = float(args.steps * args.events_per_step) * P
+        if state_digest(h) != want_digest:
+            raise SystemExit("the timed run did not end in the state of the generating pass")
+        h.close()
+        units = float(K * eps) * P
         t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
         n_multi = batch1["multi_launches"] - batch0["multi_launches"]
         n_batched = batch1["batched_arrivals"] - batch0["batched_arrivals"]
@@ -491,62 +508,81 @@ def main():
                     "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel}
         if n_multi:
             roofline["arrivals_per_multi_launch"] = n_batched / n_multi
-        return {"value": units_all / (t_ms * 1e-3), "ms_per_step": t_ms / args.steps, "launches": int(launches),
+        return {"value": units_all / (t_ms * 1e-3), "ms_per_step": t_ms / K, "launches": int(launches),
                 "roofline": roofline, "clocks": clk.summary()}
 
-    per_event = timed_region(1, 0)                       # one kernel per event
-    if args.max_batch > 1:
-        main_run = timed_region(args.max_batch, n_steps)  # multi-event fusion in the driver
-    else:
-        main_run = per_event
-    for which, idx in [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]:
-        if not np.isfinite(h.read(which, idx, 0, 4096)).all():
-            raise SystemExit("non-finite model values after the timed region")
+    per_event = timed_region(1)                          # one kernel per event
+    main_run = timed_region(args.max_batch) if args.max_batch > 1 else per_event   # multi-event fusion in the driver
     value, roofline, launches = main_run["value"], main_run["roofline"], main_run["launches"]
-    t_ms = main_run["ms_per_step"] * args.steps
+    t_ms = main_run["ms_per_step"] * K
 
-    # ---- end to end (host-resident worker results) ----
+    # ---- end to end: the same steps with the results in pinned HOST memory ----
     e2e = None
     if not args.no_e2e:
-        host_results = [torch.empty(P, dtype=wdt).pin_memory() for _ in range(wl.n_workers)]
-        for w in range(wl.n_workers):
-            host_results[w].copy_(results[w])
+        e2e_steps = max(1, min(K, 3))
+        n_e2e_arr = sum(1 for i in arrive_slots if i < e2e_steps * eps)
+        host_results = torch.empty((n_e2e_arr, P), dtype=wdt).pin_memory()
+        host_results.copy_(resident[:n_e2e_arr])
         probe = [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]
-        from paper_2506_04531_b200.inputs import trace as tr
-        e2e_steps = max(1, min(args.steps, 3))
-        base = 2 * n_steps
-        run_step(base, e2e=True, host_results=host_results, probe=probe)            # warm-up (allocates staging)
+        h = fresh_context()
         torch.cuda.synchronize(dev)
         if world > 1:
             dist.barrier()
         t0 = time.perf_counter()
         d2h = 0
-        arrivals = 0
-        for s in range(base + 1, base + 1 + e2e_steps):
-            d2h = run_step(s, e2e=True, host_results=host_results, probe=probe)
-            win = events[s * args.events_per_step:(s + 1) * args.events_per_step]
-            arrivals += int((win["kind"] == tr.ARRIVE).sum())
+        for s in range(e2e_steps):
+            win = timed_events[s * eps:(s + 1) * eps]
+            # results are copied in by the library; two staging buffers let the copy of the next result
+            # overlap the current update kernel, so up to two results are registered ahead
+            order = [k for k in range(len(win)) if int(win[k]["kind"]) == tr.ARRIVE]
+            ahead, fed = [], 0
+
+            def feed():
+                nonlocal fed
+                while fed < len(order) and len(ahead) < 2:
+                    k = order[fed]
+                    w = int(win[k]["worker"])
+                    if any(int(win[p]["worker"]) == w for p in ahead):
+                        break
+                    h.worker_delta_host(w, host_results[arrive_slots[s * eps + k]])
+                    ahead.append(k)
+                    fed += 1
+            for k in range(len(win)):
+                feed()
+                kind, l, w = int(win[k]["kind"]), int(win[k]["lps"]), int(win[k]["worker"])
+                if kind == tr.ARRIVE:
+                    assert ahead and ahead[0] == k
+                    ahead.pop(0)
+                    if h.lps_apply(l, w):
+                        h.lps_push(l)
+                elif kind == tr.GPS_RECV:
+                    h.gps_merge(l)
+                else:
+                    h.lps_pull(l)
+            # device -> host read of the step's result: a probe of the global and local models
+            d2h = sum(h.read(which, idx, 0, 1024).nbytes for which, idx in probe)
         torch.cuda.synchronize(dev)
         dt_ms = (time.perf_counter() - t0) * 1e3
-        u = float(e2e_steps * args.events_per_step) * P
+        u = float(e2e_steps * eps) * P
         dt_ms, u_all = reduce_over_ranks(dist if world > 1 else None, dt_ms, u, dev)
         e2e = {"value": u_all / (dt_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(arrivals / e2e_steps * P * (4 if wl.worker_dtype == gen.F32 else 2)),
-               "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps}
+               "h2d_bytes_per_step": int(n_e2e_arr / e2e_steps * P * wbytes), "d2h_bytes_per_step": int(d2h),
+               "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps}
         e2e["h2d_GBps"] = e2e["h2d_bytes_per_step"] / (e2e["ms_per_step"] * 1e6)   # the PCIe copy bounds this leg
+        h.close()
         del host_results
 
-    h.close()
-    del results
+    del resident, scratch
     torch.cuda.empty_cache()
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        rate, desc, spent, done = oracle_sample(wl, events, 1 << 22, args.cpu_budget_s)
+        cpu_events = wl.trace()                     # the whole configured trace: the sample stops at the time budget
+        rate, desc, spent, done = oracle_sample(wl, cpu_events, 1 << 22, args.cpu_budget_s)
         cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc + f" ({spent:.1f} s)"}
         try:
-            all_rate, n_cores = oracle_sample_all_cores(wl, events, 1 << 20, min(6.0, args.cpu_budget_s))
+            all_rate, n_cores = oracle_sample_all_cores(wl, cpu_events, 1 << 20, min(6.0, args.cpu_budget_s))
             cpu["all_cores"] = {"value": all_rate, "cores": n_cores,
                                 "sample": "one replayer per core, each on its own 1M-parameter slice, up to 6 s"}
         except Exception as e:       # the single-core figure is the baseline; this one is additional context
