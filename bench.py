@@ -470,8 +470,11 @@ def main():
             e0.record()
             for s in range(K):
                 base = s * eps
+                # streaming form: arrivals still waiting for companions at the end of a step may be fused
+                # with arrivals of the next step; everything is launched before the region ends
                 h.replay(timed_events[base:base + eps], lambda index, worker, rnd, base=base: resident[arrive_slots[base + index]],
-                         want_log=False, max_batch=max_batch)
+                         want_log=False, max_batch=max_batch, keep_queued=True)
+            h.flush()
             e1.record()
             torch.cuda.synchronize(dev)
         if world > 1:

@@ -221,6 +221,20 @@ int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, hal
 int halos_replay_batched(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                          void* user, halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch);
 
+/* Streaming form of halos_replay_batched for a queue that is fed call after call: arrivals still
+ * waiting for companions when the call returns STAY queued (their counters are already advanced, their
+ * kernels not yet launched) and may be fused with arrivals of the next call.  They are launched by the
+ * next call that needs them, by halos_flush, and by every other entry point that reads or changes
+ * the state they touch (lps_apply, lps_push, lps_pull, export/import, timing, destroy; peek and read
+ * launch the queue of the LPS or worker whose buffer is asked for).  A result
+ * returned by the producer must stay valid until the same worker's next producer call or the next
+ * halos_flush, whichever comes first. */
+int halos_replay_stream(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
+                        void* user, halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch);
+
+/* Launches every arrival that halos_replay_stream left queued. */
+int halos_flush(halos_ctx* ctx);
+
 /* Read-only device pointer to a state buffer (for inspection; valid until halos_destroy).
  * *numel = P.  Element type fp32, or worker_dtype for HALOS_BUF_THETA0. */
 int halos_peek(halos_ctx* ctx, uint32_t which, uint32_t index, const void** ptr_dev, uint64_t* numel);

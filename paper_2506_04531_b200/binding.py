@@ -35,7 +35,8 @@ EXPORTED = (
     "halos_lps_push", "halos_gps_merge", "halos_lps_pull", "halos_destroy", "halos_replay", "halos_peek",
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
     "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
-    "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards",
+    "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards", "halos_replay_stream",
+    "halos_flush",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -102,6 +103,8 @@ def load_library():
     lib.halos_replay.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32)]
     lib.halos_replay_batched.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
     lib.halos_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.halos_replay_stream.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
+    lib.halos_flush.argtypes = [vp]
     lib.halos_batch_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
     lib.halos_peek.argtypes = [vp, u32, u32, C.POINTER(vp), C.POINTER(u64)]
     lib.halos_read.argtypes = [vp, u32, u32, u64, u64, vp]
@@ -225,6 +228,7 @@ class Halos:
         if rc != OK:
             raise HalosError(rc, self._lib.halos_last_error(None).decode())
         self._keep = {}
+        self._stream_hold = []
 
     # ------------------------------------------------------------------ plumbing
     def _check(self, rc: int):
@@ -281,11 +285,13 @@ class Halos:
         self._check(self._lib.halos_lps_pull(self._h, lps))
 
     # ------------------------------------------------------------------ auxiliary
-    def replay(self, events: np.ndarray, producer: Callable, want_log: bool = True, max_batch: int = 1):
+    def replay(self, events: np.ndarray, producer: Callable, want_log: bool = True, max_batch: int = 1,
+               keep_queued: bool = False):
         """events: structured array (kind, lps, worker, pad, time_ns); producer(event_index, worker, round)
         returns a flat tensor/address or a list of per-tensor tensors.  max_batch > 1 turns on multi-event
         fusion (then a result must stay valid until the producer is called again for the same worker).
-        Returns the event log."""
+        keep_queued=True is the streaming form: arrivals still queued at the end stay queued for the next
+        call (launch them with flush()).  Returns the event log."""
         ev = np.ascontiguousarray(events)
         assert ev.dtype.itemsize == C.sizeof(Event)
         log = np.zeros(len(ev), dtype=EVENT_LOG_DTYPE) if want_log else None
@@ -309,13 +315,21 @@ class Halos:
 
         cb = PRODUCER_FN(_prod)
         failed = C.c_uint32(0)
-        rc = self._lib.halos_replay_batched(self._h, ev.ctypes.data, len(ev), cb, None,
-                                            log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch))
+        fn = self._lib.halos_replay_stream if keep_queued else self._lib.halos_replay_batched
+        if keep_queued:
+            self._stream_hold.append(hold)       # results must outlive this call
+        rc = fn(self._h, ev.ctypes.data, len(ev), cb, None,
+                log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch))
         if err:
             raise err[0]
         if rc != OK:
             raise HalosError(rc, f"event {failed.value}: " + self._lib.halos_last_error(self._h).decode())
         return log
+
+    def flush(self):
+        """Launches the arrivals that replay(..., keep_queued=True) left queued."""
+        self._check(self._lib.halos_flush(self._h))
+        self._stream_hold.clear()
 
     def peek(self, which: int, index: int = 0):
         """Zero-copy torch view of a state buffer (fp32, or int16 bit patterns for bf16 worker snapshots)."""

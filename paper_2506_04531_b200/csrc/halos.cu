@@ -51,6 +51,12 @@ struct GuardedBuffer {
     size_t bytes;    // data size
 };
 
+// An arrival whose counters are already advanced but whose kernel launch is deferred (multi-event fusion).
+struct Deferred {
+    uint32_t worker;
+    const void* flat;   // NULL: per-tensor pointer table of that worker
+};
+
 struct TimedLaunch {
     cudaEvent_t a, b;
     int kind;
@@ -89,6 +95,7 @@ struct halos_ctx {
     int stage_owner[kStageSlots] = {-1, -1};
     int stage_next = 0;
 
+    std::vector<std::vector<Deferred>> deferred;  // per LPS: arrivals accounted for, not yet launched
     std::vector<void*> owned;  // device allocations made through the allocator
     std::vector<GuardedBuffer> guards;
     uint64_t launches = 0;
@@ -379,10 +386,6 @@ int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int*
 }
 
 // ---- batched arrivals (multi-event fusion) -------------------------------------------------------
-struct Deferred {
-    uint32_t worker;
-    const void* flat;   // NULL: per-tensor pointer table of that worker
-};
 
 template <class W, int NB>
 int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push) {
@@ -438,6 +441,41 @@ int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool 
 
 int flush_deferred(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool push) {
     return c->wb == 4 ? flush_deferred_t<float>(c, lps, q, push) : flush_deferred_t<uint16_t>(c, lps, q, push);
+}
+
+// Launch everything that is still queued (a queued arrival never carries a push: those are flushed at once).
+int flush_all(halos_ctx* c) {
+    int rc = HALOS_OK;
+    for (uint32_t l = 0; l < c->deferred.size(); ++l) {
+        if (c->deferred[l].empty()) continue;
+        int rf = flush_deferred(c, l, c->deferred[l], false);
+        if (rc == HALOS_OK) rc = rf;
+    }
+    return rc;
+}
+
+// Launch what a reader of one state buffer depends on: the queue of that LPS, or of that worker's LPS if the
+// worker has an arrival queued; the GPS buffers never wait (GPS events are not deferred).
+int flush_worker(halos_ctx* c, uint32_t worker);
+int flush_for(halos_ctx* c, uint32_t which, uint32_t index) {
+    switch (which) {
+        case HALOS_BUF_THETA_L: case HALOS_BUF_M_L: case HALOS_BUF_ANCHOR: case HALOS_BUF_OUTBOX: case HALOS_BUF_INBOX:
+        case HALOS_BUF_ACC_L:
+            if (index < c->deferred.size() && !c->deferred[index].empty()) return flush_deferred(c, index, c->deferred[index], false);
+            return HALOS_OK;
+        case HALOS_BUF_THETA0:
+            return index < c->workers.size() ? flush_worker(c, index) : HALOS_OK;
+        default:
+            return HALOS_OK;
+    }
+}
+
+// Before the pointer table or the result buffer of a worker is replaced, its queued arrival must have been launched.
+int flush_worker(halos_ctx* c, uint32_t worker) {
+    std::vector<Deferred>& q = c->deferred[c->workers[worker].lps];
+    for (const Deferred& d : q)
+        if (d.worker == worker) return flush_deferred(c, c->workers[worker].lps, q, false);
+    return HALOS_OK;
 }
 
 }  // namespace
@@ -555,6 +593,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     const bool dn = cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV;
     if (dn) ok &= (c->acc_g = (float*)S(P * 4)) != nullptr;
     c->lps.resize(cfg->n_lps);
+    c->deferred.resize(cfg->n_lps);
     for (auto& s : c->lps) {
         if (!ok) break;
         ok &= (s.th = (float*)S(P * 4)) != nullptr;
@@ -620,6 +659,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
 int halos_destroy(halos_ctx* c) {
     if (!c) return HALOS_OK;
     cudaSetDevice(c->cfg.device);
+    (void)flush_all(c);
     release(c);
     delete c;
     return HALOS_OK;
@@ -631,6 +671,10 @@ int halos_worker_delta(halos_ctx* c, uint32_t worker, const void* flat, const vo
     if ((flat == nullptr) == (ptrs == nullptr)) return fail(c, HALOS_ERR_INVALID_ARG, "give exactly one of flat / pointer table");
     WorkerState& w = c->workers[worker];
     if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u already has a pending result", worker);
+    {
+        int rq = flush_worker(c, worker);   // a still-queued arrival of this worker reads its old result / table
+        if (rq != HALOS_OK) return rq;
+    }
     if (flat) {
         if (reinterpret_cast<uintptr_t>(flat) % c->wb) return fail(c, HALOS_ERR_INVALID_ARG, "thetaH not aligned to its element size");
         if (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) {
@@ -670,6 +714,10 @@ int halos_worker_delta_host(halos_ctx* c, uint32_t worker, const void* host) {
     if (worker >= c->cfg.n_workers || !host) return fail(c, HALOS_ERR_INVALID_ARG, "bad worker or null pointer");
     WorkerState& w = c->workers[worker];
     if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u already has a pending result", worker);
+    {
+        int rq = flush_worker(c, worker);
+        if (rq != HALOS_OK) return rq;
+    }
     int slot = -1;
     for (int k = 0; k < kStageSlots; ++k) {
         int s = (c->stage_next + k) % kStageSlots;
@@ -708,12 +756,18 @@ int halos_worker_delta_host(halos_ctx* c, uint32_t worker, const void* host) {
 
 int halos_lps_apply(halos_ctx* c, uint32_t lps, uint32_t worker, int* push_due) {
     if (!c) return HALOS_ERR_INVALID_ARG;
+    int rq = flush_all(c);
+    if (rq != HALOS_OK) return rq;
     return apply_impl(c, lps, worker, false, push_due);
 }
 
 int halos_lps_push(halos_ctx* c, uint32_t lps) {
     if (!c) return HALOS_ERR_INVALID_ARG;
     if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
     LpsState& s = c->lps[lps];
     if (s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u already has a round trip in flight", lps);
     CU(c, cudaSetDevice(c->cfg.device));
@@ -761,8 +815,17 @@ int halos_gps_merge(halos_ctx* c, uint32_t lps) {
     return HALOS_OK;
 }
 
+static int pull_impl(halos_ctx* c, uint32_t lps);
+
 int halos_lps_pull(halos_ctx* c, uint32_t lps) {
     if (!c) return HALOS_ERR_INVALID_ARG;
+    int rq = flush_all(c);
+    if (rq != HALOS_OK) return rq;
+    return pull_impl(c, lps);
+}
+
+// the caller has launched whatever was queued for this LPS
+static int pull_impl(halos_ctx* c, uint32_t lps) {
     if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
     LpsState& s = c->lps[lps];
     if (s.phase != HALOS_ANSWERED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Theta_i to merge", lps);
@@ -788,8 +851,8 @@ int halos_lps_pull(halos_ctx* c, uint32_t lps) {
 // the worker's snapshot; outbox_l only when it pushes) is disjoint from what events of other LPSs and
 // GPS_RECV(l) touch, so the deferred launches commute with the launches they are moved past and the
 // final state is bit-identical to the unbatched replay.
-int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
-                         halos_event_log* log, uint32_t* failed_at, uint32_t max_batch) {
+int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
+                        halos_event_log* log, uint32_t* failed_at, uint32_t max_batch) {
     if (!c) return HALOS_ERR_INVALID_ARG;
     if (n && !ev) return fail(c, HALOS_ERR_INVALID_ARG, "null event array");
     if (max_batch == 0) max_batch = 1;
@@ -797,7 +860,7 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
     if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
     const bool immediate = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV ||       // launched event by event
                            (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) != 0;
-    std::vector<std::vector<Deferred>> queue(c->cfg.n_lps);
+    std::vector<std::vector<Deferred>>& queue = c->deferred;
     int rc = HALOS_OK;
     uint32_t k = 0;
     for (; k < n && rc == HALOS_OK; ++k) {
@@ -849,7 +912,7 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
             rc = flush_deferred(c, e.lps, queue[e.lps], false);
             if (rc == HALOS_OK) {
                 if (c->lps[e.lps].phase == HALOS_ANSWERED) rec.gps_lag = c->gps_iter - c->lps[e.lps].inbox_iter;
-                rc = halos_lps_pull(c, e.lps);
+                rc = pull_impl(c, e.lps);
             }
         } else {
             rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: unknown kind %u", k, (unsigned)e.kind);
@@ -861,13 +924,24 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
             log[k] = rec;
         }
     }
-    // whatever is still queued belongs to events already accounted for: launch it
-    for (uint32_t l = 0; l < c->cfg.n_lps; ++l) {
-        int rf = flush_deferred(c, l, queue[l], false);
-        if (rc == HALOS_OK && rf != HALOS_OK) rc = rf;
+    if (rc != HALOS_OK) {
+        (void)flush_all(c);   // events before the failing one stay applied: launch what they queued
+        if (failed_at) *failed_at = k ? k - 1 : 0;
     }
-    if (rc != HALOS_OK && failed_at) *failed_at = k ? k - 1 : 0;
     return rc;
+}
+
+int halos_flush(halos_ctx* c) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    return flush_all(c);
+}
+
+int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
+                         halos_event_log* log, uint32_t* failed_at, uint32_t max_batch) {
+    int rc = halos_replay_stream(c, ev, n, producer, user, log, failed_at, max_batch);
+    if (!c) return rc;
+    int rf = flush_all(c);   // whatever is still queued belongs to events already accounted for
+    return rc != HALOS_OK ? rc : rf;
 }
 
 int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
@@ -908,6 +982,10 @@ int stream_buffer(halos_ctx* c, FILE* f, void* dev, size_t bytes, bool to_file, 
 
 int checkpoint(halos_ctx* c, const char* path, bool to_file) {
     if (!c || !path) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
     for (auto& w : c->workers)
         if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "a worker result is registered but not applied");
     CU(c, cudaSetDevice(c->cfg.device));
@@ -1010,6 +1088,10 @@ static int buffer_of(halos_ctx* c, uint32_t which, uint32_t index, const void** 
 
 int halos_peek(halos_ctx* c, uint32_t which, uint32_t index, const void** ptr_dev, uint64_t* numel) {
     if (!c || !ptr_dev) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_for(c, which, index);
+        if (rq != HALOS_OK) return rq;
+    }
     const void* p;
     uint32_t eb;
     int rc = buffer_of(c, which, index, &p, &eb);
@@ -1021,6 +1103,10 @@ int halos_peek(halos_ctx* c, uint32_t which, uint32_t index, const void** ptr_de
 
 int halos_read(halos_ctx* c, uint32_t which, uint32_t index, uint64_t offset, uint64_t count, void* dst) {
     if (!c || (!dst && count)) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_for(c, which, index);
+        if (rq != HALOS_OK) return rq;
+    }
     const void* p;
     uint32_t eb;
     int rc = buffer_of(c, which, index, &p, &eb);
@@ -1077,6 +1163,10 @@ int halos_info(halos_ctx* c, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunk
 int halos_check_guards(halos_ctx* c, int32_t* first_bad) {
     if (!c) return HALOS_ERR_INVALID_ARG;
     if (!(c->cfg.flags & HALOS_FLAG_GUARD)) return fail(c, HALOS_ERR_BAD_STATE, "context was created without HALOS_FLAG_GUARD");
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaStreamSynchronize(c->stream));
     int32_t bad = -1;
@@ -1106,6 +1196,10 @@ int halos_batch_info(halos_ctx* c, uint64_t* multi_launches, uint64_t* batched_a
 
 int halos_timing_enable(halos_ctx* c, int on) {
     if (!c) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaStreamSynchronize(c->stream));
     for (auto& t : c->timed) c->event_pool.emplace_back(t.a, t.b);
@@ -1116,6 +1210,10 @@ int halos_timing_enable(halos_ctx* c, int on) {
 
 int halos_timing_read(halos_ctx* c, uint32_t kind, uint64_t* launches, double* total_ms) {
     if (!c || kind >= HALOS_K_COUNT) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaStreamSynchronize(c->stream));
     uint64_t n = 0;

@@ -828,3 +828,54 @@ def test_config_70m_every_element():
     with cf.ThreadPoolExecutor(max_workers=cores) as ex:
         bad = [b for part in ex.map(run_slice, range(cores)) for b in part]
     assert not bad, bad[:5]
+
+
+def test_streaming_replay_keeps_batches_across_calls():
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 3])
+    worker_lps = [0, 0, 0, 0, 0, 0, 1, 1, 1, 2]
+    hp = dict(K=9, **PAPER_HP)
+    speeds = [1.0, 1.05, 1.1, 1.15, 1.2, 3.9, 1.1, 1.2, 3.3, 2.0]
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=speeds, t_profiled_ms=1.0,
+                                            n_arrivals=240, K=9))
+    dg = DeviceGenerator(lay, 29)
+
+    def make(h):
+        bufs = [torch.empty(lay.P, dtype=torch.float32, device="cuda") for _ in worker_lps]
+        return lambda index, worker, rnd: dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker])
+
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    log_ref = ref.replay(events, make(ref))
+    one = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    one.replay(events, make(one), max_batch=8)
+    st = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    prod = make(st)
+    logs = []
+    for a in range(0, len(events), 5):                       # five events per call: far shorter than a batch window
+        logs.append(st.replay(events[a:a + 5], prod, max_batch=8, keep_queued=True))
+    queued_before = st.info()["launches"]
+    st.flush()
+    cut = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    prod_cut = make(cut)
+    for a in range(0, len(events), 5):
+        cut.replay(events[a:a + 5], prod_cut, max_batch=8)   # same calls, but every call flushes
+    # streaming fuses as well as one big call and much better than calls that flush
+    assert st.info()["launches"] <= one.info()["launches"] + 1
+    assert st.info()["launches"] < 0.9 * cut.info()["launches"]
+    log_st = np.concatenate(logs)
+    for f in ("kind", "lps", "worker", "t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+        assert np.array_equal(log_ref[f], log_st[f]), f
+    for h in (one, st, cut):
+        for which in range(8):
+            n = len(worker_lps) if which == hb.BUF_THETA0 else (1 if which < 2 else 3)
+            for idx in range(n):
+                assert np.array_equal(ref.read(which, idx).view(np.uint8), h.read(which, idx).view(np.uint8)), (which, idx)
+    # any entry point that looks at the state launches what is queued
+    st2 = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    st2.replay(events[:3], make(st2), max_batch=8, keep_queued=True)
+    ref2 = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    ref2.replay(events[:3], make(ref2))
+    l0 = int(events[0]["lps"])
+    assert np.array_equal(st2.read(hb.BUF_THETA_L, l0).view(np.uint32), ref2.read(hb.BUF_THETA_L, l0).view(np.uint32))
+    for h in (ref, one, st, cut, st2, ref2):
+        h.close()
