@@ -48,10 +48,11 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {"arrive_f32": 28, "arrive_bf16": 22, "arrive_push_f32": 36, "arrive_push_bf16": 30,
                    "push": 12, "gps": 24, "pull": 16}
 
-# DRAM read+write bytes per parameter per launch, from an ncu capture of the 70M-parameter fp32
-# profiling workload (P = 70,426,624; the summary is kept with the other ncu summaries; traffic is
+# DRAM read+write bytes per parameter per launch, from ncu captures of the 70M-parameter fp32 and bf16
+# profiling workloads (P = 70,426,624; the summary is kept with the other ncu summaries; traffic is
 # proportional to P).
-DRAM_BYTES_PER_PARAM = {"arrive_f32": 27.22, "arrive_push_f32": 35.23, "gps": 23.20, "pull": 15.20}
+DRAM_BYTES_PER_PARAM = {"arrive_f32": 27.21, "arrive_push_f32": 35.23, "arrive_bf16": 21.22, "arrive_push_bf16": 29.22,
+                        "gps": 23.20, "pull": 15.22}
 
 
 # ------------------------------------------------------------------------------------ helpers
@@ -504,8 +505,8 @@ def main():
         d_bytes = kernel_bytes(dominant, dn) / dn
         achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
         tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
-        if dominant == "arrive_multi" and wname == "f32" and n_multi:
-            tpp = 15.24 + 12.0 * n_batched / n_multi     # measured: model and momentum cross HBM once per batch
+        if dominant == "arrive_multi" and n_multi:
+            tpp = 15.24 + 3.0 * wbytes * n_batched / n_multi   # measured: model and momentum cross HBM once per batch
         roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak,
                     "unit": "GB/s", "frac": achieved / peak, "traffic": (tpp * P if tpp else None),
                     "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel}
