@@ -3,6 +3,8 @@
 #include "halos.h"
 #include "halos_kernels.cuh"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -191,11 +193,16 @@ void build_chunks(halos_ctx* c, uint32_t chunk_elems) {
     c->tensor_chunk_begin[c->tensor_numel.size()] = (uint32_t)c->chunks.size();
 }
 
+// Brackets one kernel launch: an NVTX range named after the kernel kind (visible to profilers, free
+// otherwise) and, while timing is enabled, a pair of CUDA events on the context's stream.
+const char* const kKindNames[HALOS_K_COUNT] = {"halos:arrive", "halos:arrive+push", "halos:push", "halos:gps",
+                                               "halos:pull", "halos:arrive_multi"};
 struct Timer {
     halos_ctx* c;
     cudaEvent_t a = nullptr, b = nullptr;
     int kind;
     Timer(halos_ctx* c_, int kind_) : c(c_), kind(kind_) {
+        nvtxRangePushA(kKindNames[kind]);
         if (!c->timing) return;
         if (!c->event_pool.empty()) {
             a = c->event_pool.back().first;
@@ -209,6 +216,7 @@ struct Timer {
         cudaEventRecord(a, c->stream);
     }
     void stop() {
+        nvtxRangePop();
         if (!a) return;
         cudaEventRecord(b, c->stream);
         c->timed.push_back(TimedLaunch{a, b, kind});
