@@ -879,3 +879,35 @@ def test_streaming_replay_keeps_batches_across_calls():
     assert np.array_equal(st2.read(hb.BUF_THETA_L, l0).view(np.uint32), ref2.read(hb.BUF_THETA_L, l0).view(np.uint32))
     for h in (ref, one, st, cut, st2, ref2):
         h.close()
+
+
+def test_replay_stops_at_the_first_bad_event_and_keeps_what_came_before():
+    P = 4096
+    init = torch.linspace(-1, 1, P, device="cuda")
+    good = hb.Halos(init, [0, 0, 1], K=3, **PAPER_HP)
+    bad = hb.Halos(init, [0, 0, 1], K=3, **PAPER_HP)
+    res = [init + 0.01 * (w + 1) for w in range(3)]
+    ev = np.zeros(6, dtype=tr.EVENT_DTYPE)
+    ev["kind"] = [tr.ARRIVE, tr.ARRIVE, tr.ARRIVE, tr.PULL, tr.ARRIVE, tr.ARRIVE]
+    ev["lps"] = [0, 1, 0, 1, 0, 0]
+    ev["worker"] = [0, 2, 1, 0, 0, 1]
+    good.replay(ev[:3], lambda i, w, r: res[w], max_batch=4)
+    with pytest.raises(hb.HalosError) as e:                  # event 3: PULL for an LPS that never pushed
+        bad.replay(ev, lambda i, w, r: res[w], max_batch=4)
+    assert e.value.status == hb.ERR_BAD_STATE and "event 3" in str(e.value)
+    for l in (0, 1):
+        assert bad.counters(l) == good.counters(l)
+        assert np.array_equal(bad.read(hb.BUF_THETA_L, l), good.read(hb.BUF_THETA_L, l))
+    # a failing producer aborts the replay and its exception reaches the caller
+    def broken(i, w, r):
+        raise KeyError("no result for this worker")
+    with pytest.raises(KeyError):
+        bad.replay(ev[4:5], broken)
+    assert bad.counters(0) == good.counters(0) and not bad.worker_info(0)["pending"]
+    ev2 = ev[:1].copy()
+    ev2["lps"] = 9
+    with pytest.raises(hb.HalosError) as e:
+        bad.replay(ev2, lambda i, w, r: res[w])
+    assert e.value.status == hb.ERR_INVALID_ARG
+    good.close()
+    bad.close()
