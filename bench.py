@@ -305,7 +305,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "410m", "70m_f32_small"])
+    ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "160m_dn", "410m", "70m_f32_small"])
     ap.add_argument("--events-per-step", type=int, default=0,
                     help="events per step; 0 = 128, reduced so that the results of all timed steps fit in HBM")
     ap.add_argument("--no-e2e", action="store_true")

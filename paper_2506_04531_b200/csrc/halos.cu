@@ -57,6 +57,7 @@ struct GuardedBuffer {
 struct Deferred {
     uint32_t worker;
     const void* flat;   // NULL: per-tensor pointer table of that worker
+    bool refresh;       // delayed Nesterov: this update refreshes the momentum (decided when it was accounted for)
 };
 
 struct TimedLaunch {
@@ -224,7 +225,7 @@ struct Timer {
 };
 
 template <class W>
-int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
+int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known) {
     ArriveDnArgs<W> a;
     a.h_flat = (const W*)flat;
     a.h_ptrs = flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)widx * c->tensor_numel.size());
@@ -239,7 +240,8 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
     a.beta = c->cfg.beta_l;
     a.inv_n = 1.0f / (float)c->cfg.delay_l;
     a.eps_n = c->cfg.eta_l * a.inv_n;
-    const bool refresh = ((s.t + 1) % c->cfg.delay_l) == 0;   // s.t is advanced after the launch
+    // refresh_known < 0: the launch precedes the counter update, so this is update number s.t + 1
+    const bool refresh = refresh_known >= 0 ? refresh_known != 0 : ((s.t + 1) % c->cfg.delay_l) == 0;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
@@ -257,8 +259,8 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
 }
 
 template <class W>
-int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat) {
-    if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat);
+int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known = -1) {
+    if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat, refresh_known);
     if (w.pending == PEND_DELTA) {
         ArriveDeltaArgs<W> d{w.delta, (W*)w.th0, s.th, s.ml, s.anchor, s.outbox, c->cfg.eta_l, c->cfg.beta_l, 1.0f - c->cfg.beta_l};
         const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
@@ -396,7 +398,49 @@ int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int*
 // ---- batched arrivals (multi-event fusion) -------------------------------------------------------
 
 template <class W, int NB>
+int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool push) {
+    ArriveMultiDnArgs<W> a;
+    const size_t nt = c->tensor_numel.size();
+    a.refresh_mask = 0;
+    for (int j = 0; j < kMaxBatch; ++j) {
+        const int k = j < NB ? j : 0;
+        a.h_flat[j] = (const W*)d[k].flat;
+        a.h_ptrs[j] = d[k].flat ? nullptr : (const W* const*)(c->d_ptr_tables + (size_t)d[k].worker * nt);
+        a.th0[j] = (W*)c->workers[d[k].worker].th0;
+        if (j < NB && d[j].refresh) a.refresh_mask |= 1u << j;
+    }
+    a.tensor_off = c->d_tensor_off;
+    a.th = s.th;
+    a.ml = s.ml;
+    a.acc = s.acc;
+    a.anchor = s.anchor;
+    a.outbox = s.outbox;
+    a.eps = c->cfg.eta_l;
+    a.beta = c->cfg.beta_l;
+    a.inv_n = 1.0f / (float)c->cfg.delay_l;
+    a.eps_n = c->cfg.eta_l * a.inv_n;
+    constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
+    const dim3 grid((unsigned)c->chunks.size()), block(TPB);
+    const bool any = a.refresh_mask != 0;
+    Timer tm(c, HALOS_K_ARRIVE_MULTI);
+    if (any) {
+        if (push) arrive_multi_dn_kernel<W, NB, true, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_multi_dn_kernel<W, NB, true, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    } else {
+        if (push) arrive_multi_dn_kernel<W, NB, false, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        else arrive_multi_dn_kernel<W, NB, false, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    }
+    tm.stop();
+    c->launches++;
+    c->batched_arrivals += NB;
+    c->multi_launches++;
+    CU(c, cudaGetLastError());
+    return HALOS_OK;
+}
+
+template <class W, int NB>
 int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push) {
+    if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_multi_dn<W, NB>(c, s, d, push);
     ArriveMultiArgs<W> a;
     const size_t nt = c->tensor_numel.size();
     for (int j = 0; j < kMaxBatch; ++j) {
@@ -433,7 +477,7 @@ int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool 
     int rc = HALOS_OK;
     CU(c, cudaSetDevice(c->cfg.device));
     switch (q.size()) {
-        case 1: rc = launch_arrive<W>(c, s, c->workers[q[0].worker], q[0].worker, push, q[0].flat); break;
+        case 1: rc = launch_arrive<W>(c, s, c->workers[q[0].worker], q[0].worker, push, q[0].flat, q[0].refresh ? 1 : 0); break;
         case 2: rc = launch_arrive_multi<W, 2>(c, s, q.data(), push); break;
         case 3: rc = launch_arrive_multi<W, 3>(c, s, q.data(), push); break;
         case 4: rc = launch_arrive_multi<W, 4>(c, s, q.data(), push); break;
@@ -866,8 +910,7 @@ int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_p
     if (max_batch == 0) max_batch = 1;
     if (max_batch > (uint32_t)kMaxBatch) max_batch = kMaxBatch;
     if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
-    const bool immediate = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV ||       // launched event by event
-                           (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) != 0;
+    const bool immediate = (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) != 0;   // launched event by event
     std::vector<std::vector<Deferred>>& queue = c->deferred;
     int rc = HALOS_OK;
     uint32_t k = 0;
@@ -906,7 +949,9 @@ int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_p
                     if (w.pending == PEND_STAGED || immediate) {
                         rc = apply_impl(c, e.lps, e.worker, true, nullptr);   // host-staged results are not deferred
                     } else {
-                        q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr});
+                        const bool refresh = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV &&
+                                             ((c->lps[e.lps].t + 1) % c->cfg.delay_l) == 0;
+                        q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr, refresh});
                         rec.fused = (uint8_t)(q.size() > 1 || push);
                         apply_commit(c, e.lps, e.worker, push);
                         if (push || q.size() >= max_batch) rc = flush_deferred(c, e.lps, q, push);

@@ -569,6 +569,109 @@ gps_dn_kernel(const Chunk* __restrict__ chunks, GpsDnArgs a) {
 }
 
 // =====================================================================================================
+// ARRIVE x NB with the delayed-Nesterov optimizer: the model and the accumulator cross HBM once per
+// batch; the momentum only if one of the batched updates is a refresh (bit j of refresh_mask).
+// =====================================================================================================
+template <class W>
+struct ArriveMultiDnArgs {
+    const W* h_flat[kMaxBatch];
+    const W* const* h_ptrs[kMaxBatch];
+    W* th0[kMaxBatch];
+    const unsigned long long* tensor_off;
+    float* th;
+    float* ml;
+    float* acc;
+    const float* anchor;
+    float* outbox;
+    float eps, beta, inv_n, eps_n;
+    uint32_t refresh_mask;
+};
+
+template <class W, int NB, bool ANYREF, bool PUSH, bool STREAM, int VE, int TPB>
+__global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
+arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a) {
+    using T = WTraits<W>;
+    const Chunk c = chunks[blockIdx.x];
+    const W* h[NB];
+    W* s0[NB];
+    bool vec_ok = (c.begin % VE) == 0;
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        h[j] = a.h_flat[j] ? a.h_flat[j] + c.begin : a.h_ptrs[j][c.tensor] + (c.begin - a.tensor_off[c.tensor]);
+        s0[j] = a.th0[j] + c.begin;
+        vec_ok = vec_ok && ((reinterpret_cast<uintptr_t>(h[j]) % (VE * sizeof(W))) == 0);
+    }
+    float* th = a.th + c.begin;
+    float* ml = a.ml + c.begin;
+    float* ac = a.acc + c.begin;
+    const float* an = PUSH ? a.anchor + c.begin : nullptr;
+    float* ob = PUSH ? a.outbox + c.begin : nullptr;
+    const float eps = a.eps, beta = a.beta, inv_n = a.inv_n, eps_n = a.eps_n;
+    const uint32_t mask = a.refresh_mask;
+    uint32_t done = 0;
+    if (vec_ok) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += TPB) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vh[NB], vs[NB], vx, vc, vm, va;
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                vh[j] = T::template load<VE, STREAM>(h[j] + o);
+                vs[j] = T::template load<VE, STREAM>(s0[j] + o);
+            }
+            vx = ldf<VE, STREAM>(th + o);
+            vc = ldf<VE, STREAM>(ac + o);
+            if (ANYREF) vm = ldf<VE, STREAM>(ml + o);
+            if (PUSH) va = ldf<VE, STREAM>(an + o);
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const bool refresh = ANYREF && ((mask >> j) & 1u);   // uniform over the grid
+#pragma unroll
+                for (int e = 0; e < VE; ++e) {
+                    const float d = __fsub_rn(vh[j].v[e], vs[j].v[e]);
+                    if (refresh) {
+                        float m = vm.v[e];
+                        delayed_nesterov<true>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
+                        vm.v[e] = m;
+                    } else {
+                        float m = 0.f;
+                        delayed_nesterov<false>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
+                    }
+                }
+                T::template store<VE, STREAM>(s0[j] + o, vx);
+            }
+            stf<VE, STREAM>(th + o, vx);
+            stf<VE, STREAM>(ac + o, vc);
+            if (ANYREF) stf<VE, STREAM>(ml + o, vm);
+            if (PUSH) {
+                FVec<VE> D;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                stf<VE, STREAM>(ob + o, D);
+            }
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t i = done + threadIdx.x; i < c.count; i += TPB) {
+        float x = th[i], acc = ac[i], m = ANYREF ? ml[i] : 0.f;
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
+            if (ANYREF && ((mask >> j) & 1u)) delayed_nesterov<true>(x, m, acc, d, eps, beta, inv_n, eps_n);
+            else {
+                float unused = 0.f;
+                delayed_nesterov<false>(x, unused, acc, d, eps, beta, inv_n, eps_n);
+            }
+            T::store1(s0[j] + i, x);
+        }
+        th[i] = x;
+        ac[i] = acc;
+        if (ANYREF) ml[i] = m;
+        if (PUSH) ob[i] = __fsub_rn(x, an[i]);
+    }
+}
+
+// =====================================================================================================
 // Materialised delta (HALOS_FLAG_MATERIALISE_DELTA): the worker-side subtraction of Alg. 1 line 25 runs
 // when the result is handed over, delta (fp32) is kept in a context buffer, and the caller's theta_H is
 // free again as soon as that kernel has been enqueued.  The LPS update then reads delta instead of

@@ -38,6 +38,9 @@ class Workload:
     lps_gbps: Optional[Sequence[float]] = None        # LPS -> GPS link of each LPS (default: by region l % 4)
     dyn_updates: bool = False
     bandwidth_scale: float = 1.0
+    optimizer: int = 0                # 0: the update rule the paper defines; 1: delayed Nesterov (its experiments)
+    delay_l: int = 1
+    delay_g: int = 1
 
     @property
     def worker_lps(self) -> List[int]:
@@ -63,12 +66,15 @@ class Workload:
             lps_gbps=self.lps_gbps, dyn_updates=self.dyn_updates, bandwidth_scale=self.bandwidth_scale))
 
     def hyper(self) -> dict:
-        return dict(eta_l=self.eta_l, beta_l=self.beta_l, eta_g=self.eta_g, beta_g=self.beta_g,
-                    alpha=self.alpha, K=self.K)
+        hp = dict(eta_l=self.eta_l, beta_l=self.beta_l, eta_g=self.eta_g, beta_g=self.beta_g,
+                  alpha=self.alpha, K=self.K)
+        if self.optimizer:
+            hp.update(optimizer=self.optimizer, delay_l=self.delay_l, delay_g=self.delay_g)
+        return hp
 
 
 def workload(name: str) -> Workload:
-    """toy | toy_k4 | 70m | 160m | 410m | 70m_f32_small | paper_cluster | paper_cluster_small |
+    """toy | toy_k4 | 70m | 160m | 160m_dn | 410m | 70m_f32_small | paper_cluster | paper_cluster_small |
     hetero_grouping_small  (hyperparameters: the paper's selected values)."""
     if name == "toy":
         return Workload("toy", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1)
@@ -81,6 +87,11 @@ def workload(name: str) -> Workload:
     if name == "410m":
         return Workload("410m", named_layout("410m"), 32, 4, gen.F32, 1589.7, 2000, seed=4,
                         slow_region_factor=3.0)
+    if name == "160m_dn":
+        # the 160M configuration under the optimizer and the selected values of the paper's experiments:
+        # delayed Nesterov with d_l = 16, eta_l = 16 x 0.2, d_g = 2, eta_g = 2 x 0.15
+        return Workload("160m_dn", named_layout("160m"), 16, 4, gen.F32, 623.0, 2000, seed=3,
+                        eta_l=3.2, eta_g=0.3, optimizer=1, delay_l=16, delay_g=2)
     if name == "paper_cluster":
         # the paper's own simulated cluster: 4 regions x 4 workers with its 16 worker speeds, one LPS
         # per region, dynamic local updates, 160M layout

@@ -553,8 +553,8 @@ def test_delayed_nesterov_replay_and_checkpoint(tmp_path):
     ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, **hp)
     run(ref, events, 1)
     a = hb.Halos(dg.theta_init(), worker_lps, lay.numel, **hp)
-    run(a, events[:37], 4)                 # batching requested: this optimizer still launches event by event
-    assert a.batch_info()["multi_launches"] == 0
+    run(a, events[:37], 4)                 # batched (fused delayed-Nesterov launches) up to the checkpoint
+    assert a.batch_info()["multi_launches"] > 0
     a.export_file(tmp_path / "dn.ckpt")
     a.close()
     b = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, **hp)
@@ -911,3 +911,36 @@ def test_replay_stops_at_the_first_bad_event_and_keeps_what_came_before():
     assert e.value.status == hb.ERR_INVALID_ARG
     good.close()
     bad.close()
+
+
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+@pytest.mark.parametrize("delay_l", [1, 3, 16])
+def test_batched_replay_with_delayed_nesterov(wdt, delay_l):
+    """Fused launches under the delayed-Nesterov optimizer: refreshes may fall anywhere inside a batch."""
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192, 8191, 3])
+    worker_lps = [0, 0, 0, 0, 0, 0, 0, 0, 1, 1, 1, 2]
+    hp = dict(DN_HP, K=11, delay_l=delay_l)
+    speeds = [1.0, 1.05, 1.1, 1.15, 1.2, 1.25, 1.3, 3.9, 1.1, 1.2, 3.3, 2.0]
+    events = tr.generate_trace(tr.TraceSpec(P=lay.P, worker_lps=worker_lps, speeds=speeds, t_profiled_ms=1.0,
+                                            n_arrivals=300, K=11))
+    dg = DeviceGenerator(lay, 31)
+    tdt = torch.float32 if wdt == gen.F32 else torch.int16
+
+    def make(h):
+        bufs = [torch.empty(lay.P, dtype=tdt, device="cuda") for _ in worker_lps]
+        return lambda index, worker, rnd: dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker],
+                                                           worker_dtype=wdt)
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, chunk_elems=1024, **hp)
+    log_ref = ref.replay(events, make(ref))
+    bat = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, chunk_elems=1024, **hp)
+    log_bat = bat.replay(events, make(bat), max_batch=8)
+    assert bat.batch_info()["multi_launches"] > 10
+    for which in list(range(8)) + [hb.BUF_ACC_L, hb.BUF_ACC_G]:
+        n = len(worker_lps) if which == hb.BUF_THETA0 else (1 if which in (0, 1, hb.BUF_ACC_G) else 3)
+        for idx in range(n):
+            assert np.array_equal(ref.read(which, idx).view(np.uint8), bat.read(which, idx).view(np.uint8)), (which, idx)
+    for f in ("t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+        assert np.array_equal(log_ref[f], log_bat[f]), f
+    ref.close()
+    bat.close()
