@@ -79,6 +79,8 @@ struct halos_ctx {
     cudaStream_t copy_stream = nullptr;
 
     Chunk* d_chunks = nullptr;
+    Chunk* d_chunks_rev = nullptr;  // the same table in reverse order
+    bool flip = false;              // direction of the next launch
     unsigned long long* d_tensor_off = nullptr;
     uint32_t* d_tensor_chunk_begin = nullptr;
     const void** d_ptr_tables = nullptr;  // [n_workers][n_tensors]
@@ -198,6 +200,16 @@ void build_chunks(halos_ctx* c, uint32_t chunk_elems) {
 // otherwise) and, while timing is enabled, a pair of CUDA events on the context's stream.
 const char* const kKindNames[HALOS_K_COUNT] = {"halos:arrive", "halos:arrive+push", "halos:push", "halos:gps",
                                                "halos:pull", "halos:arrive_multi"};
+// Chunk table of the next launch.  Consecutive launches walk the buffers in opposite directions, so that
+// a launch starts on the lines its predecessor touched last, which are still in L2 (worth 1-3% on
+// buffers several times the size of L2).  Statistics index their partial sums by table position and
+// always use the forward table.
+const Chunk* next_table(halos_ctx* c) {
+    if (c->cfg.flags & HALOS_FLAG_STATS) return c->d_chunks;
+    c->flip = !c->flip;
+    return c->flip ? c->d_chunks : c->d_chunks_rev;
+}
+
 struct Timer {
     halos_ctx* c;
     cudaEvent_t a = nullptr, b = nullptr;
@@ -246,11 +258,11 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
     if (refresh) {
-        if (push) arrive_dn_kernel<W, true, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_dn_kernel<W, true, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (push) arrive_dn_kernel<W, true, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_dn_kernel<W, true, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     } else {
-        if (push) arrive_dn_kernel<W, false, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_dn_kernel<W, false, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (push) arrive_dn_kernel<W, false, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_dn_kernel<W, false, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     }
     tm.stop();
     c->launches++;
@@ -266,8 +278,8 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
         const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
         if (grid.x == 0) return HALOS_OK;
         Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
-        if (push) arrive_delta_kernel<W, true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, d);
-        else arrive_delta_kernel<W, false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, d);
+        if (push) arrive_delta_kernel<W, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), d);
+        else arrive_delta_kernel<W, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), d);
         tm.stop();
         c->launches++;
         CU(c, cudaGetLastError());
@@ -293,11 +305,11 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
     if (push) {
-        if (stats) arrive_kernel<W, true, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_kernel<W, true, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (stats) arrive_kernel<W, true, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_kernel<W, true, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     } else {
-        if (stats) arrive_kernel<W, false, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_kernel<W, false, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (stats) arrive_kernel<W, false, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_kernel<W, false, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     }
     tm.stop();
     c->launches++;
@@ -326,7 +338,7 @@ int launch_delta_t(halos_ctx* c, uint32_t worker, const void* flat) {
     a.th0 = (const W*)w.th0;
     a.delta = w.delta;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
-    if (grid.x) delta_kernel<W, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (grid.x) delta_kernel<W, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     c->launches++;
     CU(c, cudaGetLastError());
     return HALOS_OK;
@@ -424,11 +436,11 @@ int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool pu
     const bool any = a.refresh_mask != 0;
     Timer tm(c, HALOS_K_ARRIVE_MULTI);
     if (any) {
-        if (push) arrive_multi_dn_kernel<W, NB, true, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_multi_dn_kernel<W, NB, true, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (push) arrive_multi_dn_kernel<W, NB, true, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_multi_dn_kernel<W, NB, true, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
     } else {
-        if (push) arrive_multi_dn_kernel<W, NB, false, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else arrive_multi_dn_kernel<W, NB, false, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (push) arrive_multi_dn_kernel<W, NB, false, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else arrive_multi_dn_kernel<W, NB, false, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
     }
     tm.stop();
     c->launches++;
@@ -460,8 +472,8 @@ int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push)
     constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     Timer tm(c, HALOS_K_ARRIVE_MULTI);
-    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-    else arrive_multi_kernel<W, NB, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+    else arrive_multi_kernel<W, NB, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
     tm.stop();
     c->launches++;
     c->batched_arrivals += NB;
@@ -631,6 +643,7 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     };
     bool ok = true;
     ok &= (c->d_chunks = (Chunk*)A(nc * sizeof(Chunk))) != nullptr;
+    ok &= (c->d_chunks_rev = (Chunk*)A(nc * sizeof(Chunk))) != nullptr;
     ok &= (c->d_tensor_off = (unsigned long long*)A((nt + 1) * 8)) != nullptr;
     ok &= (c->d_tensor_chunk_begin = (uint32_t*)A((nt + 1) * 4)) != nullptr;
     ok &= (c->d_ptr_tables = (const void**)A((size_t)cfg->n_workers * nt * 8)) != nullptr;
@@ -679,6 +692,8 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
 
     cudaStream_t st = c->stream;
     CUC(cudaMemcpyAsync(c->d_chunks, c->chunks.data(), nc * sizeof(Chunk), cudaMemcpyHostToDevice, st));
+    std::vector<Chunk> reversed(c->chunks.rbegin(), c->chunks.rend());
+    CUC(cudaMemcpyAsync(c->d_chunks_rev, reversed.data(), nc * sizeof(Chunk), cudaMemcpyHostToDevice, st));
     CUC(cudaMemcpyAsync(c->d_tensor_off, c->tensor_off.data(), (nt + 1) * 8, cudaMemcpyHostToDevice, st));
     CUC(cudaMemcpyAsync(c->d_tensor_chunk_begin, c->tensor_chunk_begin.data(), (nt + 1) * 4, cudaMemcpyHostToDevice, st));
     if (c->d_stats) CUC(cudaMemsetAsync(c->d_stats, 0, (size_t)3 * cfg->n_lps * nt * 8, st));
@@ -827,8 +842,8 @@ int halos_lps_push(halos_ctx* c, uint32_t lps) {
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
     Timer tm(c, HALOS_K_PUSH);
-    if (stats) push_kernel<true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-    else push_kernel<false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    if (stats) push_kernel<true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+    else push_kernel<false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
@@ -852,11 +867,11 @@ int halos_gps_merge(halos_ctx* c, uint32_t lps) {
     if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) {
         const float inv_n = 1.0f / (float)c->cfg.delay_g;
         GpsDnArgs a{s.outbox, c->Theta, c->Mg, c->acc_g, s.inbox, c->cfg.eta_g, c->cfg.beta_g, inv_n, c->cfg.eta_g * inv_n};
-        if (((c->gps_iter + 1) % c->cfg.delay_g) == 0) gps_dn_kernel<true, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
-        else gps_dn_kernel<false, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        if (((c->gps_iter + 1) % c->cfg.delay_g) == 0) gps_dn_kernel<true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+        else gps_dn_kernel<false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     } else {
         GpsArgs a{s.outbox, c->Theta, c->Mg, s.inbox, c->cfg.eta_g, c->cfg.beta_g, 1.0f - c->cfg.beta_g};
-        gps_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+        gps_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     }
     tm.stop();
     c->launches++;
@@ -885,7 +900,7 @@ static int pull_impl(halos_ctx* c, uint32_t lps) {
     PullArgs a{s.th, s.inbox, s.anchor, c->cfg.alpha, 1.0f - c->cfg.alpha};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     Timer tm(c, HALOS_K_PULL);
-    pull_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(c->d_chunks, a);
+    pull_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
