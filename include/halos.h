@@ -55,8 +55,8 @@ enum { HALOS_F32 = 0, HALOS_BF16 = 1 };
 /* Server-side optimizer.
  * HALOS_OPT_PAPER: the ModelUpdate rule the paper defines (Appendix E); the default.
  * HALOS_OPT_DELAYED_NESTEROV: the optimizer the paper's experiments used ("delayed Nesterov", cited from
- * the Async-Local-SGD work, never defined in the paper; its hyperparameter table only says that the
- * rule "effectively divides the learning rate by the delay interval").  Reading implemented, per server
+ * the Async-Local-SGD work, never defined in the paper; the footnote of its hyperparameter table in
+ * Appendix D only states that the rule scales the step by 1/delay).  Reading implemented, per server
  * with delay n, rate eps (= eta_l / eta_g), accumulator acc, k = number of updates seen so far:
  *     acc += d                                            every update (d = displacement)
  *     k mod n != 0:   x += (eps/n) d                      momentum untouched
@@ -260,7 +260,9 @@ int halos_info(halos_ctx* ctx, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chu
 
 /* Checkpoint / resume.  halos_export_file writes the whole state (every buffer, all counters and
  * phases) to a file; halos_import_file loads it into a context that was created with the same
- * shape (P, tensors, servers, workers, worker_dtype; checked) and replaces its state, so that a
+ * shape (P, tensors, servers, workers, worker_dtype, optimizer) and the same hyperparameters (K, eta_l,
+ * beta_l, eta_g, beta_g, alpha bit for bit, and delay_l / delay_g under delayed Nesterov) -- all checked,
+ * a mismatch is INVALID_ARG and leaves the context untouched -- and replaces its state, so that a
  * replay continued after export -> destroy -> create -> import equals the uninterrupted replay bit
  * for bit.  Both wait for the stream.  BAD_STATE if any worker result is registered but not yet
  * applied (borrowed caller memory cannot be checkpointed); INVALID_ARG on I/O errors or a file
@@ -305,14 +307,19 @@ int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double*
  * three enables the vector path; sqnorm_dev points to one double).  The reduction scratch is a fixed
  * 512 KB array inside the library, present on every GPU that loads it until the process exits, which
  * caps n at HALOS_NOALLOC_MAX_ELEMS: larger n returns HALOS_ERR_UNSUPPORTED and touches nothing.
- * The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine) and enqueues
- * two kernels on `stream` (cudaStream_t, NULL = legacy default stream); it does not wait for them.
- * The first call on each device looks up the scratch array's device address (cudaGetSymbolAddress)
- * and should therefore be made before any stream capture begins.  All calls share the scratch,
+ * Once warmed up, a call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine) and
+ * enqueues two kernels on `stream` (cudaStream_t, NULL = legacy default stream); it does not wait for them.
+ * Warm-up: the FIRST call on each device may create that device's primary context, loads the two kernels
+ * and the scratch array with them (the runtime takes device memory for this) and looks up the array's
+ * device address (cudaGetSymbolAddress).  Make that call -- n = 0 is enough -- at start-up, while
+ * allocation is still allowed and before any stream capture begins; later calls on that device touch no
+ * allocator.  Every call makes `device` the calling thread's current CUDA device and leaves it so.
+ * All calls share the scratch,
  * which keeps the previous call's partial sums; each call overwrites every slot it later reads, so
  * nothing needs clearing, but calls that overlap on the GPU race on it: keep them on one stream or
  * otherwise serialised.  Returns HALOS_OK, HALOS_ERR_UNSUPPORTED (n too large),
- * HALOS_ERR_INVALID_ARG (null/misaligned pointer, bad device) or HALOS_ERR_CUDA. */
+ * HALOS_ERR_INVALID_ARG (null pointer, array not 4-byte aligned, sqnorm_dev not 8-byte aligned, bad
+ * device; checked on the host before anything is launched) or HALOS_ERR_CUDA. */
 #define HALOS_NOALLOC_MAX_ELEMS (1ull << 29)
 int halos_push_noalloc(int32_t device, void* stream, const float* theta_dev, const float* anchor_dev,
                        float* Delta_dev, uint64_t n, double* sqnorm_dev);

@@ -33,8 +33,8 @@
 //
 // Optional optimizer OPT_DELAYED_NESTEROV.  The paper's experiments replace ModelUpdate by the
 // "delayed Nesterov" optimizer of the Async-Local-SGD work it cites, but never define it; the only
-// property it states is that the rule "effectively divides the learning rate by the delay interval"
-// (hyperparameter table, Appendix D).  The reading implemented here, per server with delay d,
+// property it states (footnote of the hyperparameter table, Appendix D) is that the rule scales the
+// step by 1/delay.  The reading implemented here, per server with delay d,
 // rate eps, an accumulator acc and n = number of updates seen so far:
 //     acc += g                                        every update
 //     n mod d != 0:  theta -= (eps/d) g               momentum untouched

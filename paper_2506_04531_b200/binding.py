@@ -12,11 +12,8 @@ from typing import Callable, Optional, Sequence
 
 import numpy as np
 
-import os
-
 _PKG = Path(__file__).resolve().parent
-# HALOS_B200_LIB points at an alternative build of the same library (kernel tuning experiments).
-LIB_PATH = Path(os.environ.get("HALOS_B200_LIB", _PKG / "libhalos_b200.so"))
+LIB_PATH = _PKG / "libhalos_b200.so"
 
 OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED = range(6)
 F32, BF16 = 0, 1
@@ -228,9 +225,14 @@ class Halos:
         if rc != OK:
             raise HalosError(rc, self._lib.halos_last_error(None).decode())
         self._keep = {}
-        self._stream_hold = []
+        self._stream_hold = {}
 
     # ------------------------------------------------------------------ plumbing
+    def _mark_in_use(self, x):
+        """Tells the caching allocator that a CUDA tensor is read by work on the context's stream."""
+        if hasattr(x, "record_stream") and getattr(x, "is_cuda", False):
+            x.record_stream(self._stream)
+
     def _check(self, rc: int):
         if rc != OK:
             raise HalosError(rc, self._lib.halos_last_error(self._h).decode())
@@ -295,7 +297,11 @@ class Halos:
         ev = np.ascontiguousarray(events)
         assert ev.dtype.itemsize == C.sizeof(Event)
         log = np.zeros(len(ev), dtype=EVENT_LOG_DTYPE) if want_log else None
-        hold = {}
+        # Results are borrowed by the library until the kernels that read them have run.  They are kept per
+        # worker: a worker's entry is replaced at its next producer call (the library has launched its previous
+        # arrival by then) and every tensor is marked as in use on the context's stream, so that the caching
+        # allocator does not hand its block to another stream while an enqueued kernel still reads it.
+        hold = self._stream_hold if keep_queued else {}
         err = []
 
         def _prod(_user, index, worker, rnd, flat_out, ptrs_out):
@@ -303,11 +309,14 @@ class Halos:
                 r = producer(int(index), int(worker), int(rnd))
                 if isinstance(r, (list, tuple)):
                     arr = (C.c_void_p * self.n_tensors)(*[_ptr(t) for t in r])
-                    hold[(worker, "p")] = (r, arr)
+                    hold[worker] = (r, arr)
                     ptrs_out[0] = C.cast(arr, C.POINTER(C.c_void_p))
+                    for t in r:
+                        self._mark_in_use(t)
                 else:
                     hold[worker] = r
                     flat_out[0] = _ptr(r)
+                    self._mark_in_use(r)
                 return 0
             except Exception as e:  # surfaced after the call returns
                 err.append(e)
@@ -316,8 +325,6 @@ class Halos:
         cb = PRODUCER_FN(_prod)
         failed = C.c_uint32(0)
         fn = self._lib.halos_replay_stream if keep_queued else self._lib.halos_replay_batched
-        if keep_queued:
-            self._stream_hold.append(hold)       # results must outlive this call
         rc = fn(self._h, ev.ctypes.data, len(ev), cb, None,
                 log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch))
         if err:

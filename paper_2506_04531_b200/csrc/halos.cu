@@ -349,15 +349,23 @@ int launch_delta(halos_ctx* c, uint32_t worker, const void* flat) {
 
 // Host-side part of an arrival (Alg. 1 lines 10 and 13): argument/state checks and counter updates.
 // *due = this arrival completes a window of K; *push = the caller wants Delta formed with it.
-int apply_check(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, bool* due, bool* push) {
+// The part of the check that does not need a registered result (the replay driver runs it BEFORE it asks
+// the producer for one, so that a refused event leaves no borrowed pointer behind).
+int arrival_check(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, bool* due, bool* push) {
     if (lps >= c->cfg.n_lps || worker >= c->cfg.n_workers) return fail(c, HALOS_ERR_INVALID_ARG, "lps/worker out of range");
     WorkerState& w = c->workers[worker];
     if (w.lps != lps) return fail(c, HALOS_ERR_INVALID_ARG, "worker %u does not belong to LPS %u", worker, lps);
-    if (w.pending == PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u has no pending result", worker);
     LpsState& s = c->lps[lps];
     *due = (s.t + 1 - s.t_last == c->cfg.K);
     *push = fuse_push && *due;
     if (*push && s.phase != HALOS_IDLE) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u: push due while a round trip is in flight", lps);
+    return HALOS_OK;
+}
+
+int apply_check(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, bool* due, bool* push) {
+    int rc = arrival_check(c, lps, worker, fuse_push, due, push);
+    if (rc != HALOS_OK) return rc;
+    if (c->workers[worker].pending == PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "worker %u has no pending result", worker);
     return HALOS_OK;
 }
 
@@ -951,13 +959,15 @@ int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_p
                     }
                 const void* flat = nullptr;
                 const void* const* ptrs = nullptr;
+                bool due = false, push = false;
+                // membership and the state of the round trip are checked before the producer is asked, so
+                // that a refused event registers nothing
+                if (rc == HALOS_OK) rc = arrival_check(c, e.lps, e.worker, true, &due, &push);
                 if (rc == HALOS_OK && w.pending == PEND_NONE) {
                     if (producer(user, k, e.worker, w.round, &flat, &ptrs) != 0)
                         rc = fail(c, HALOS_ERR_INVALID_ARG, "event %u: producer failed", k);
                     else rc = halos_worker_delta(c, e.worker, flat, ptrs);
                 }
-                bool due = false, push = false;
-                if (rc == HALOS_OK) rc = apply_check(c, e.lps, e.worker, true, &due, &push);
                 if (rc == HALOS_OK && (w.pending == PEND_STAGED || immediate) && !q.empty()) rc = flush_deferred(c, e.lps, q, false);
                 if (rc == HALOS_OK) {
                     rec.worker_staleness = c->lps[e.lps].t - w.sched_t;
@@ -1027,6 +1037,7 @@ struct CkptHeader {
     float eta_l, beta_l, eta_g, beta_g, alpha;
     uint32_t optimizer;
     uint64_t gps_iter;
+    uint32_t delay_l, delay_g;
 };
 struct CkptLps { uint64_t t, t_last, t_push, inbox_iter; int32_t phase; int32_t pad; };
 struct CkptWorker { uint64_t round, sched_t; };
@@ -1073,11 +1084,13 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
     std::vector<CkptWorker> ws(c->workers.size());
     if (to_file) {
         std::memcpy(h.magic, "HALOSCK1", 8);
-        h.version = 1; h.wb = c->wb; h.P = c->P;
+        h.version = 2; h.wb = c->wb; h.P = c->P;
         h.n_lps = c->cfg.n_lps; h.n_workers = c->cfg.n_workers; h.n_tensors = c->cfg.n_tensors; h.K = c->cfg.K;
         h.eta_l = c->cfg.eta_l; h.beta_l = c->cfg.beta_l; h.eta_g = c->cfg.eta_g; h.beta_g = c->cfg.beta_g; h.alpha = c->cfg.alpha;
         h.gps_iter = c->gps_iter;
         h.optimizer = c->cfg.optimizer;
+        h.delay_l = c->cfg.delay_l;
+        h.delay_g = c->cfg.delay_g;
         for (size_t l = 0; l < ls.size(); ++l)
             ls[l] = CkptLps{c->lps[l].t, c->lps[l].t_last, c->lps[l].t_push, c->lps[l].inbox_iter, c->lps[l].phase, 0};
         for (size_t w = 0; w < ws.size(); ++w) ws[w] = CkptWorker{c->workers[w].round, c->workers[w].sched_t};
@@ -1086,11 +1099,18 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
             rc = fail(c, HALOS_ERR_INVALID_ARG, "short write to checkpoint file");
     } else {
         std::vector<uint64_t> numel(c->tensor_numel.size());
-        if (fread(&h, sizeof h, 1, f) != 1 || std::memcmp(h.magic, "HALOSCK1", 8) != 0 || h.version != 1)
-            rc = fail(c, HALOS_ERR_INVALID_ARG, "not a checkpoint file of this library");
+        if (fread(&h, sizeof h, 1, f) != 1 || std::memcmp(h.magic, "HALOSCK1", 8) != 0 || h.version != 2)
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "not a checkpoint file of this library (or of another version)");
         else if (h.P != c->P || h.wb != c->wb || h.n_lps != c->cfg.n_lps || h.n_workers != c->cfg.n_workers || h.n_tensors != c->cfg.n_tensors ||
                  h.optimizer != c->cfg.optimizer)
             rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint shape does not match this context");
+        // A run resumed under other hyperparameters is another run: the window length and the delays fix
+        // WHEN pushes and momentum refreshes happen, the rates and momenta fix every later value.
+        else if (h.K != c->cfg.K || std::memcmp(&h.eta_l, &c->cfg.eta_l, 4) || std::memcmp(&h.beta_l, &c->cfg.beta_l, 4) ||
+                 std::memcmp(&h.eta_g, &c->cfg.eta_g, 4) || std::memcmp(&h.beta_g, &c->cfg.beta_g, 4) ||
+                 std::memcmp(&h.alpha, &c->cfg.alpha, 4) ||
+                 (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV && (h.delay_l != c->cfg.delay_l || h.delay_g != c->cfg.delay_g)))
+            rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint hyperparameters (K, rates, momenta, alpha, delays) differ from this context's");
         else if (fread(numel.data(), 8, numel.size(), f) != numel.size() || numel != c->tensor_numel)
             rc = fail(c, HALOS_ERR_INVALID_ARG, "checkpoint tensor sizes do not match this context");
         else if (fread(ls.data(), sizeof(CkptLps), ls.size(), f) != ls.size() || fread(ws.data(), sizeof(CkptWorker), ws.size(), f) != ws.size())

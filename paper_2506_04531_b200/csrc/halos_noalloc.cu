@@ -121,6 +121,7 @@ extern "C" int halos_push_noalloc(int32_t device, void* stream, const float* the
     if ((reinterpret_cast<uintptr_t>(theta_dev) | reinterpret_cast<uintptr_t>(anchor_dev) |
          reinterpret_cast<uintptr_t>(Delta_dev)) & 3)
         return HALOS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(sqnorm_dev) & 7) return HALOS_ERR_INVALID_ARG;  // a double is stored through it
     if (cudaSetDevice(device) != cudaSuccess) {
         (void)cudaGetLastError();
         return HALOS_ERR_CUDA;
@@ -133,6 +134,14 @@ extern "C" int halos_push_noalloc(int32_t device, void* stream, const float* the
         if (!g_partials_addr[device]) {
             double* p = nullptr;
             if (cudaGetSymbolAddress((void**)&p, g_partials) != cudaSuccess || !p) {
+                (void)cudaGetLastError();
+                return HALOS_ERR_CUDA;
+            }
+            // Load both kernels (and with them the module that holds the scratch array) now, so that
+            // this first call is the only one that can make the runtime take device memory.
+            cudaFuncAttributes fa;
+            if (cudaFuncGetAttributes(&fa, push_flat_kernel) != cudaSuccess ||
+                cudaFuncGetAttributes(&fa, sum_partials_kernel) != cudaSuccess) {
                 (void)cudaGetLastError();
                 return HALOS_ERR_CUDA;
             }

@@ -110,8 +110,9 @@ def workload(name: str) -> Workload:
                         fixed_speeds=PAPER_WORKER_SPEEDS, fixed_worker_lps=wl_map,
                         lps_gbps=[GBPS_TO_GPS_REGION[r] for r in region_of_lps], bandwidth_scale=2.0)
     if name == "70m_f32_small":
-        # profiling case: 70M layout, fp32 copies, 4 workers on 1 LPS (~4 GB on the device, every
-        # buffer still larger than L2); K=8 so that pushes, GPS updates and merges occur early
+        # small-memory configuration (~4 GB on the device): the 70M layout with fp32 copies, 4 workers on
+        # 1 LPS; every buffer is still larger than L2, and K = 8 makes pushes, GPS updates and merges
+        # occur within the first few events.  For GPUs with little free memory and for counter captures.
         return Workload("70m_f32_small", named_layout("70m"), 4, 1, gen.F32, 238.4, 200, seed=6, K=8)
     raise KeyError(name)
 

@@ -399,6 +399,14 @@ def test_checkpoint_resume_is_bit_identical(tmp_path, wdt):
     with pytest.raises(hb.HalosError) as e:
         other.import_file(path)
     assert e.value.status == hb.ERR_INVALID_ARG
+    # ... and so is a context with the same shape but other hyperparameters (a different run)
+    for change in (dict(K=5), dict(eta_l=0.25), dict(beta_g=0.4), dict(alpha=0.5)):
+        odd = hb.Halos(torch.ones(lay.P, device="cuda"), worker_lps, lay.numel, worker_dtype=wdt, **dict(hp, **change))
+        with pytest.raises(hb.HalosError) as e:
+            odd.import_file(path)
+        assert e.value.status == hb.ERR_INVALID_ARG and "hyperparameters" in str(e.value)
+        assert odd.counters(0)["t"] == 0 and float(odd.read(hb.BUF_THETA_L, 0, 0, 8).min()) == 1.0   # untouched
+        odd.close()
     # pending results cannot be checkpointed
     b.worker_delta(0, scratch)
     with pytest.raises(hb.HalosError) as e:
@@ -565,6 +573,11 @@ def test_delayed_nesterov_replay_and_checkpoint(tmp_path):
     for l in (0, 1):
         for which in (hb.BUF_THETA_L, hb.BUF_M_L, hb.BUF_ACC_L, hb.BUF_ANCHOR):
             assert np.array_equal(ref.read(which, l).view(np.uint32), b.read(which, l).view(np.uint32))
+    other_delay = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, **dict(hp, delay_l=4))
+    with pytest.raises(hb.HalosError) as e:
+        other_delay.import_file(tmp_path / "dn.ckpt")  # another refresh schedule: refused
+    assert e.value.status == hb.ERR_INVALID_ARG
+    other_delay.close()
     plain = hb.Halos(torch.zeros(lay.P, device="cuda"), worker_lps, lay.numel, K=4)
     with pytest.raises(hb.HalosError):
         plain.import_file(tmp_path / "dn.ckpt")       # other optimizer: refused
@@ -909,6 +922,22 @@ def test_replay_stops_at_the_first_bad_event_and_keeps_what_came_before():
     with pytest.raises(hb.HalosError) as e:
         bad.replay(ev2, lambda i, w, r: res[w])
     assert e.value.status == hb.ERR_INVALID_ARG
+    # an arrival that names a worker of another LPS is refused BEFORE the producer is asked: nothing is
+    # registered, so no borrowed pointer outlives the failed call
+    ev3 = ev[:1].copy()
+    ev3["lps"], ev3["worker"] = 1, 0
+    asked = []
+    with pytest.raises(hb.HalosError) as e:
+        bad.replay(ev3, lambda i, w, r: asked.append(w) or res[w])
+    assert e.value.status == hb.ERR_INVALID_ARG and not asked
+    assert not bad.worker_info(0)["pending"]
+    # the same for an arrival that would close a window while the previous round trip is still in flight
+    late = hb.Halos(init, [0, 0, 1], K=1, **PAPER_HP)
+    late.replay(ev[:1], lambda i, w, r: res[w])              # K = 1: this arrival pushes
+    with pytest.raises(hb.HalosError) as e:
+        late.replay(ev[2:3], lambda i, w, r: asked.append(w) or res[w])
+    assert e.value.status == hb.ERR_BAD_STATE and not asked and not late.worker_info(1)["pending"]
+    late.close()
     good.close()
     bad.close()
 

@@ -491,3 +491,55 @@ def test_bf16_worker_snapshots():
     np.testing.assert_allclose(o.buffer("th", 0), ref, rtol=2e-7, atol=1e-9)
     np.testing.assert_array_equal(o.buffer("th0", 0), to_bf16(o.buffer("th", 0)))
     np.testing.assert_array_equal(o.buffer("th0", 1), to_bf16(th_init))      # the other worker keeps its stale start
+
+
+# ----------------------------------------------------------------------------------------------
+# Bookkeeping: the worker's staleness (LPS updates applied since it was last scheduled, Alg. 1
+# lines 10 and 12: the worker is handed theta_t right after update t) counted from the trace alone
+# ----------------------------------------------------------------------------------------------
+def _staleness_from_trace(events):
+    """For every ARRIVE: how many arrivals its LPS processed after this worker's previous arrival
+    (all earlier ones for a first arrival: every worker starts from the initial model, t = 0)."""
+    out = []
+    for n, ev in enumerate(events):
+        if int(ev["kind"]) != tr.ARRIVE:
+            continue
+        l, w = int(ev["lps"]), int(ev["worker"])
+        prev = max([k for k in range(n) if int(events[k]["kind"]) == tr.ARRIVE and int(events[k]["worker"]) == w], default=-1)
+        out.append(sum(1 for k in range(prev + 1, n) if int(events[k]["kind"]) == tr.ARRIVE and int(events[k]["lps"]) == l))
+    return out
+
+
+def test_worker_staleness_bookkeeping():
+    # the worked 12-event example: arrivals A0 A2 A1 A0 . A2 . . A1 . A0 with w0, w1 at LPS 0 and w2 at LPS 1
+    worker_lps = [0, 0, 1]
+    ev = np.zeros(12, dtype=tr.EVENT_DTYPE)
+    for n, tok in enumerate(_TRACE_R7):
+        kind = {"A": tr.ARRIVE, "G": tr.GPS_RECV, "P": tr.PULL}[tok[0]]
+        ev[n]["kind"] = kind
+        ev[n]["worker"] = int(tok[1]) if kind == tr.ARRIVE else 0
+        ev[n]["lps"] = worker_lps[int(tok[1])] if kind == tr.ARRIVE else int(tok[1])
+    assert _staleness_from_trace(ev) == [0, 0, 1, 1, 0, 1, 1]          # by hand from the order above
+    cases = [(ev, worker_lps, 2)]
+    for seed, wl, K in ((3, [0, 0, 0, 1, 1], 3), (4, [0, 1, 2, 2, 1, 0, 0], 2)):
+        cases.append((tr.random_trace(wl, 150, K, seed), wl, K))
+    wl = [0, 0, 0, 1, 1, 1]
+    cases.append((tr.generate_trace(tr.TraceSpec(P=1000, worker_lps=wl, speeds=[1, 1.3, 3.7, 2, 2.2, 4], t_profiled_ms=1.0,
+                                                 n_arrivals=120, K=5)), wl, 5))
+    for events, wl, K in cases:
+        o = HalosOracle(np.zeros(3, np.float32), wl, K=K)
+        got = []
+        for e in events:
+            kind, l, w = int(e["kind"]), int(e["lps"]), int(e["worker"])
+            if kind == tr.ARRIVE:
+                got.append(o.counters(l)["t"] - o.worker_info(w)["sched_t"])
+                o.arrive(w, np.zeros(3, np.float32))
+                assert o.worker_info(w)["sched_t"] == o.counters(l)["t"]
+            elif kind == tr.GPS_RECV:
+                o.gps_recv(l)
+            else:
+                o.pull(l)
+        assert got == _staleness_from_trace(events)
+        assert [o.worker_info(w)["round"] for w in range(len(wl))] == \
+            [int(((events["kind"] == tr.ARRIVE) & (events["worker"] == w)).sum()) for w in range(len(wl))]
+        o.close()

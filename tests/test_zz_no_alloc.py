@@ -5,7 +5,10 @@ pools, start-up-only allocation policies), so its reduction scratch is a fixed a
 library that all calls share.  The test calls it twice in a row through the C ABI -- first on a
 large vector, then on a smaller, different one, so that stale partial sums of the first call would
 show up in the second -- and compares Delta bit for bit and the squared norm within the tolerance
-the statistics tests use.  It lives in a file of its own that sorts last, so a run that stops at the
+the statistics tests use: against the regular push, and against a host computation that involves
+no CUDA code (fp32 subtraction in numpy, squares summed in fp64), so that a mistake shared by the
+two CUDA paths cannot hide.  It also checks that a warmed-up call leaves the amount of free device
+memory unchanged and that a misaligned result pointer is refused on the host.  It lives in a file of its own that sorts last, so a run that stops at the
 first failure has already finished every other test; it builds its own inputs and also passes alone.
 """
 from __future__ import annotations
@@ -43,14 +46,25 @@ def test_push_noalloc_twice_in_a_row():
     build.build()
     big = _pushed_context(3_000_003, seed=11, n_arrivals=2)      # ragged tail, 367 chunks
     small = _pushed_context(70_001, seed=12, n_arrivals=3)       # 9 chunks: most slots keep the first call's sums
+    warm = torch.zeros(1, dtype=torch.float64, device="cuda")
+    assert hb.push_noalloc(big[0], big[1], big[0], warm, n=0) == hb.OK     # start-up call: loads kernels and scratch
+    torch.cuda.synchronize()
     for theta, anchor, want_Delta, want_sq in (big, small):
         out = torch.full_like(theta, float("nan"))
         sq = torch.full((1,), float("nan"), dtype=torch.float64, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         assert hb.push_noalloc(theta, anchor, out, sq) == hb.OK
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before          # nothing was allocated on the device
         assert np.array_equal(out.cpu().numpy().view(np.uint32), want_Delta.view(np.uint32))
         assert want_sq > 0
         assert abs(float(sq.item()) - want_sq) <= STATS_RTOL * want_sq
+        # the same two results from the host alone
+        host_Delta = theta.cpu().numpy() - anchor.cpu().numpy()     # fp32, one rounding per element
+        assert np.array_equal(out.cpu().numpy().view(np.uint32), host_Delta.view(np.uint32))
+        host_sq = float(np.sum(host_Delta.astype(np.float64) ** 2))
+        assert abs(float(sq.item()) - host_sq) <= STATS_RTOL * host_sq
     # unaligned views take the scalar path and give the same answer
     theta, anchor, want_Delta, want_sq = small
     pad = lambda t: torch.cat([t.new_zeros(1), t])[1:]
@@ -60,6 +74,11 @@ def test_push_noalloc_twice_in_a_row():
     torch.cuda.synchronize()
     assert np.array_equal(out.cpu().numpy().view(np.uint32), want_Delta.view(np.uint32))
     assert abs(float(sq.item()) - want_sq) <= STATS_RTOL * want_sq
+    # a result pointer that cannot hold a double is refused before anything is launched
+    two = torch.full((2,), 3.0, dtype=torch.float64, device="cuda")
+    assert hb.push_noalloc(theta, anchor, out, two.data_ptr() + 4) == hb.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert two.tolist() == [3.0, 3.0]
     # empty input: defined result, and sizes beyond the fixed scratch are refused up front
     assert hb.push_noalloc(theta, anchor, out, sq, n=0) == hb.OK
     torch.cuda.synchronize()
