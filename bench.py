@@ -46,7 +46,7 @@ if str(ROOT) not in sys.path:
 METRIC = "params_updated_per_sec"
 UNIT = "params/s"
 BYTES_PER_PARAM = {"arrive_f32": 28, "arrive_bf16": 22, "arrive_push_f32": 36, "arrive_push_bf16": 30,
-                   "push": 12, "gps": 24, "pull": 16}
+                   "push": 12, "gps": 24, "pull": 16, "gps_pull": 36}
 
 # DRAM read+write bytes per parameter per launch, from ncu captures of the 70M-parameter fp32 and bf16
 # profiling workloads (P = 70,426,624; the summary is kept with the other ncu summaries; traffic is

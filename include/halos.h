@@ -66,7 +66,9 @@ enum { HALOS_OPT_PAPER = 0, HALOS_OPT_DELAYED_NESTEROV = 1 };
 
 /* flags */
 enum {
-    HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta, theta_t (arrive) and Delta (push) */
+    HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta, theta_t (arrive) and Delta (push); formed in
+                                      registers by the update kernels, in every mode (fused launches, both optimizers,
+                                      materialised deltas); needs chunk_elems <= 8192 */
     HALOS_FLAG_GUARD = 2u,         /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
     HALOS_FLAG_MATERIALISE_DELTA = 4u  /* halos_worker_delta forms delta (fp32) into a context buffer at once, so the
                                           borrow of theta_H ends when that call has been enqueued; costs one 4P
@@ -165,6 +167,13 @@ int halos_gps_merge(halos_ctx* ctx, uint32_t lps);
  * BAD_STATE unless the GPS has answered this LPS. */
 int halos_lps_pull(halos_ctx* ctx, uint32_t lps);
 
+/* Alg. 1 lines 2-4 directly followed by lines 17-20 for the same LPS, as one launch: exactly
+ * halos_gps_merge(lps) then halos_lps_pull(lps) -- same state afterwards, bit for bit, inbox included --
+ * with Theta_i merged from registers (36 instead of 40 bytes of traffic per parameter).  For a queue in
+ * which the answer of the GPS is the very next message this LPS processes (Sec. 4.1: one queue per
+ * server, processed in order).  BAD_STATE unless lps has pushed. */
+int halos_gps_merge_pull(halos_ctx* ctx, uint32_t lps);
+
 /* Synchronises the stream and frees everything the context owns.  NULL is accepted. */
 int halos_destroy(halos_ctx* ctx);
 
@@ -203,7 +212,8 @@ typedef int (*halos_producer_fn)(void* user, uint32_t event_index, uint32_t work
                                  const void** flat_dev, const void* const** ptrs_host);
 
 /* Replays events[0..n) in order: ARRIVE = worker_delta + lps_apply (+ lps_push when the window of
- * K closes, fused into the same launch), GPS_RECV = gps_merge, PULL = lps_pull.  log_host (may be
+ * K closes, fused into the same launch), GPS_RECV = gps_merge, PULL = lps_pull (with max_batch > 1, a
+ * GPS_RECV directly followed by the PULL of the same LPS runs as halos_gps_merge_pull).  log_host (may be
  * NULL) receives one record per event.  Stops at the first failing event: returns its status and
  * writes its index to *failed_at (may be NULL); events before it stay applied. */
 int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
@@ -216,8 +226,9 @@ int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, hal
  * log and the producer calls still follow trace order; only kernel launches are deferred, past events
  * that touch disjoint buffers.  Consequence for the producer: a result it returned must stay valid
  * until the producer is called again for the SAME worker or the replay returns (with halos_replay it
- * only has to survive until the next producer call).  max_batch <= 1 behaves like halos_replay;
- * contexts with HALOS_FLAG_STATS are never batched. */
+ * only has to survive until the next producer call).  max_batch <= 1 behaves like halos_replay.
+ * Statistics (HALOS_FLAG_STATS) are kept per arrival inside fused launches and equal those of the
+ * unfused replay bit for bit (arrivals whose tensors differ in vector alignment are not fused). */
 int halos_replay_batched(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                          void* user, halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch);
 
@@ -252,8 +263,18 @@ int halos_worker_info(halos_ctx* ctx, uint32_t worker, uint64_t* info_host);
 
 /* Per-tensor squared norms (needs HALOS_FLAG_STATS): what = 0: sum delta^2 of the last
  * halos_lps_apply of this LPS; what = 1: sum Delta^2 of its last halos_lps_push; what = 2: sum theta_t^2 of
- * its model right after that last halos_lps_apply.  Waits for the stream.  out_host: [n_tensors] doubles. */
+ * its model right after that last halos_lps_apply.  After a fused launch "last" is the last arrival of the
+ * batch.  The sums are reduced in a fixed order that depends on neither the launch configuration nor the
+ * number of fused arrivals.  Waits for the stream.  out_host: [n_tensors] doubles. */
 int halos_stats(halos_ctx* ctx, uint32_t what, uint32_t lps, double* out_host);
+
+/* Per-arrival statistics log (needs HALOS_FLAG_STATS).  log_dev: caller-owned device array of
+ * capacity_records records of 3 * n_tensors doubles; from now on the r-th arrival accounted for on this
+ * context (r from 0, in trace order, however its launch is fused or deferred) fills record r with
+ * [sum delta^2 per tensor | sum theta_t^2 per tensor | sum Delta^2 per tensor (zeros unless the arrival
+ * closed a window and its push was fused)] in stream order; arrivals beyond the capacity are not recorded.
+ * NULL / 0 detaches.  The array is borrowed until detached or the context is destroyed. */
+int halos_stats_log(halos_ctx* ctx, double* log_dev, uint64_t capacity_records);
 
 /* Number of parameters P, tensors, scheduler chunks, and kernels launched so far. */
 int halos_info(halos_ctx* ctx, uint64_t* P, uint32_t* n_tensors, uint32_t* n_chunks, uint64_t* launches);
@@ -290,7 +311,8 @@ enum {
     HALOS_K_GPS = 3,          /* global momentum update + Theta_i snapshot */
     HALOS_K_PULL = 4,         /* merge + anchor reset */
     HALOS_K_ARRIVE_MULTI = 5, /* 2-8 arrivals at one LPS in one pass (halos_replay_batched) */
-    HALOS_K_COUNT = 6
+    HALOS_K_GPS_PULL = 6,     /* GPS update + merge into the same LPS in one pass (halos_gps_merge_pull) */
+    HALOS_K_COUNT = 7
 };
 int halos_timing_enable(halos_ctx* ctx, int on);
 int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double* total_ms);

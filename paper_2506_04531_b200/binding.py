@@ -24,8 +24,8 @@ IDLE, PUSHED, ANSWERED = 0, 1, 2
 BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0, BUF_ACC_L, BUF_ACC_G = range(10)
 OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1
 EV_ARRIVE, EV_GPS_RECV, EV_PULL = 0, 1, 2
-K_ARRIVE, K_ARRIVE_PUSH, K_PUSH, K_GPS, K_PULL, K_ARRIVE_MULTI = range(6)
-KERNEL_NAMES = ("arrive", "arrive_push", "push", "gps", "pull", "arrive_multi")
+K_ARRIVE, K_ARRIVE_PUSH, K_PUSH, K_GPS, K_PULL, K_ARRIVE_MULTI, K_GPS_PULL = range(7)
+KERNEL_NAMES = ("arrive", "arrive_push", "push", "gps", "pull", "arrive_multi", "gps_pull")
 
 EXPORTED = (
     "halos_default_config", "halos_create", "halos_worker_delta", "halos_worker_delta_host", "halos_lps_apply",
@@ -33,7 +33,7 @@ EXPORTED = (
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
     "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
     "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards", "halos_replay_stream",
-    "halos_flush",
+    "halos_flush", "halos_gps_merge_pull", "halos_stats_log",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -96,6 +96,8 @@ def load_library():
     lib.halos_lps_push.argtypes = [vp, u32]
     lib.halos_gps_merge.argtypes = [vp, u32]
     lib.halos_lps_pull.argtypes = [vp, u32]
+    lib.halos_gps_merge_pull.argtypes = [vp, u32]
+    lib.halos_stats_log.argtypes = [vp, vp, u64]
     lib.halos_destroy.argtypes = [vp]
     lib.halos_replay.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32)]
     lib.halos_replay_batched.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
@@ -286,6 +288,10 @@ class Halos:
     def lps_pull(self, lps: int):
         self._check(self._lib.halos_lps_pull(self._h, lps))
 
+    def gps_merge_pull(self, lps: int):
+        """gps_merge(lps) directly followed by lps_pull(lps), as one launch."""
+        self._check(self._lib.halos_gps_merge_pull(self._h, lps))
+
     # ------------------------------------------------------------------ auxiliary
     def replay(self, events: np.ndarray, producer: Callable, want_log: bool = True, max_batch: int = 1,
                keep_queued: bool = False):
@@ -371,6 +377,16 @@ class Halos:
         out = np.empty(self.n_tensors, dtype=np.float64)
         self._check(self._lib.halos_stats(self._h, what, lps, out.ctypes.data))
         return out
+
+    def stats_log(self, log=None):
+        """Attaches a float64 CUDA tensor of shape (records, 3, n_tensors) as the per-arrival statistics log
+        (None detaches); the tensor is kept alive until it is replaced."""
+        if log is None:
+            self._check(self._lib.halos_stats_log(self._h, None, 0))
+        else:
+            assert log.is_cuda and log.is_contiguous() and log.dim() == 3 and tuple(log.shape[1:]) == (3, self.n_tensors)
+            self._check(self._lib.halos_stats_log(self._h, log.data_ptr(), int(log.shape[0])))
+        self._stats_log = log
 
     def info(self) -> dict:
         P, nt, nc, nl = C.c_uint64(), C.c_uint32(), C.c_uint32(), C.c_uint64()

@@ -44,6 +44,7 @@ struct WorkerState {
     uint64_t round = 0;    // arrivals applied so far
     uint64_t sched_t = 0;  // LPS counter when last scheduled
     cudaEvent_t table_copied = nullptr;  // guards reuse of the pinned pointer-table slot
+    std::vector<uint8_t> vec_aligned;    // statistics contexts: per tensor, does the pending result allow the vector path
 };
 
 constexpr size_t kGuardBytes = 256;
@@ -58,6 +59,7 @@ struct Deferred {
     uint32_t worker;
     const void* flat;   // NULL: per-tensor pointer table of that worker
     bool refresh;       // delayed Nesterov: this update refreshes the momentum (decided when it was accounted for)
+    uint64_t seq;       // record of this arrival in the statistics log
 };
 
 struct TimedLaunch {
@@ -87,6 +89,9 @@ struct halos_ctx {
     const void** h_ptr_tables = nullptr;  // pinned mirror
     double *d_partial_delta = nullptr, *d_partial_Delta = nullptr, *d_partial_theta = nullptr;
     double* d_stats = nullptr;  // [3][n_lps][n_tensors]
+    double* stats_log = nullptr;        // caller-owned device log of per-arrival statistics (halos_stats_log)
+    uint64_t stats_log_capacity = 0;    // in records of 3 n_tensors doubles
+    uint64_t stats_seq = 0;             // arrivals accounted for since the log was attached
 
     float *Theta = nullptr, *Mg = nullptr;
     float* acc_g = nullptr;  // delayed Nesterov only
@@ -199,7 +204,7 @@ void build_chunks(halos_ctx* c, uint32_t chunk_elems) {
 // Brackets one kernel launch: an NVTX range named after the kernel kind (visible to profilers, free
 // otherwise) and, while timing is enabled, a pair of CUDA events on the context's stream.
 const char* const kKindNames[HALOS_K_COUNT] = {"halos:arrive", "halos:arrive+push", "halos:push", "halos:gps",
-                                               "halos:pull", "halos:arrive_multi"};
+                                               "halos:pull", "halos:arrive_multi", "halos:gps+pull"};
 // Chunk table of the next launch.  Consecutive launches walk the buffers in opposite directions, so that
 // a launch starts on the lines its predecessor touched last, which are still in L2 (worth 1-3% on
 // buffers several times the size of L2).  Statistics index their partial sums by table position and
@@ -236,6 +241,20 @@ struct Timer {
     }
 };
 
+// Launch helpers pick the template instance from run-time booleans.
+#define HALOS_PICK2(b0, b1, CALL)                     \
+    do {                                              \
+        if (b0) {                                     \
+            if (b1) { CALL(true, true); }             \
+            else { CALL(true, false); }               \
+        } else {                                      \
+            if (b1) { CALL(false, true); }            \
+            else { CALL(false, false); }              \
+        }                                             \
+    } while (0)
+
+inline bool stats_on(const halos_ctx* c) { return (c->cfg.flags & HALOS_FLAG_STATS) != 0; }
+
 template <class W>
 int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known) {
     ArriveDnArgs<W> a;
@@ -248,6 +267,9 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
     a.acc = s.acc;
     a.anchor = s.anchor;
     a.outbox = s.outbox;
+    a.partial_delta = c->d_partial_delta;
+    a.partial_Delta = c->d_partial_Delta;
+    a.partial_theta = c->d_partial_theta;
     a.eps = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.inv_n = 1.0f / (float)c->cfg.delay_l;
@@ -257,12 +279,15 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
-    if (refresh) {
-        if (push) arrive_dn_kernel<W, true, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_dn_kernel<W, true, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+    const Chunk* table = next_table(c);
+    if (stats_on(c)) {
+#define CALL(R, P) arrive_dn_kernel<W, R, P, true, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a)
+        HALOS_PICK2(refresh, push, CALL);
+#undef CALL
     } else {
-        if (push) arrive_dn_kernel<W, false, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_dn_kernel<W, false, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
+#define CALL(R, P) arrive_dn_kernel<W, R, P, false, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a)
+        HALOS_PICK2(refresh, push, CALL);
+#undef CALL
     }
     tm.stop();
     c->launches++;
@@ -273,13 +298,17 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
 template <class W>
 int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known = -1) {
     if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat, refresh_known);
+    const bool stats = stats_on(c);
     if (w.pending == PEND_DELTA) {
-        ArriveDeltaArgs<W> d{w.delta, (W*)w.th0, s.th, s.ml, s.anchor, s.outbox, c->cfg.eta_l, c->cfg.beta_l, 1.0f - c->cfg.beta_l};
+        ArriveDeltaArgs<W> d{w.delta, (W*)w.th0, s.th, s.ml, s.anchor, s.outbox, c->cfg.eta_l, c->cfg.beta_l, 1.0f - c->cfg.beta_l,
+                             c->d_partial_delta, c->d_partial_Delta, c->d_partial_theta};
         const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
         if (grid.x == 0) return HALOS_OK;
         Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
-        if (push) arrive_delta_kernel<W, true, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), d);
-        else arrive_delta_kernel<W, false, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), d);
+        const Chunk* table = next_table(c);
+#define CALL(P, S) arrive_delta_kernel<W, P, S, kStream, kVE><<<grid, block, 0, c->stream>>>(table, d)
+        HALOS_PICK2(push, stats, CALL);
+#undef CALL
         tm.stop();
         c->launches++;
         CU(c, cudaGetLastError());
@@ -300,28 +329,37 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
     a.eta = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.omb = 1.0f - c->cfg.beta_l;
-    const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     if (grid.x == 0) return HALOS_OK;
     Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
-    if (push) {
-        if (stats) arrive_kernel<W, true, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_kernel<W, true, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-    } else {
-        if (stats) arrive_kernel<W, false, true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_kernel<W, false, false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
-    }
+    const Chunk* table = next_table(c);
+#define CALL(P, S) arrive_kernel<W, P, S, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a)
+    HALOS_PICK2(push, stats, CALL);
+#undef CALL
     tm.stop();
     c->launches++;
     CU(c, cudaGetLastError());
     return HALOS_OK;
 }
 
-int finalize_stats(halos_ctx* c, uint32_t what, uint32_t lps) {
-    const uint32_t nt = (uint32_t)c->tensor_numel.size();
-    double* out = c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt;
-    const double* partial = what == 0 ? c->d_partial_delta : what == 1 ? c->d_partial_Delta : c->d_partial_theta;
-    stats_finalize_kernel<<<nt, 32, 0, c->stream>>>(partial, c->d_tensor_chunk_begin, out, nt);
+// Per-tensor statistics of the nb arrivals of the launch just enqueued; seq[j] = log record of arrival j.
+int finalize_stats(halos_ctx* c, uint32_t lps, uint32_t nb, bool push, const uint64_t* seq) {
+    StatsFinalizeArgs a;
+    a.partial_delta = c->d_partial_delta;
+    a.partial_theta = c->d_partial_theta;
+    a.partial_Delta = c->d_partial_Delta;
+    a.tensor_chunk_begin = c->d_tensor_chunk_begin;
+    a.last = c->d_stats;
+    a.log = c->stats_log;
+    a.log_capacity = c->stats_log_capacity;
+    for (uint32_t j = 0; j < (uint32_t)kMaxBatch; ++j) a.seq[j] = j < nb ? seq[j] : ~0ull;
+    a.n_chunks = (uint32_t)c->chunks.size();
+    a.n_tensors = (uint32_t)c->tensor_numel.size();
+    a.n_lps = c->cfg.n_lps;
+    a.lps = lps;
+    a.nb = nb;
+    a.push = push ? 1 : 0;
+    stats_finalize_kernel<<<dim3(a.n_tensors, nb, 3), 32, 0, c->stream>>>(a);
     c->launches++;
     CU(c, cudaGetLastError());
     return HALOS_OK;
@@ -405,11 +443,8 @@ int apply_impl(halos_ctx* c, uint32_t lps, uint32_t worker, bool fuse_push, int*
         CU(c, cudaEventRecord(c->stage_free[w.slot], c->stream));
         c->stage_owner[w.slot] = -1;
     }
-    if (c->cfg.flags & HALOS_FLAG_STATS) {
-        if ((rc = finalize_stats(c, 0, lps)) != HALOS_OK) return rc;
-        if ((rc = finalize_stats(c, 2, lps)) != HALOS_OK) return rc;
-        if (push && (rc = finalize_stats(c, 1, lps)) != HALOS_OK) return rc;
-    }
+    if (stats_on(c) && (rc = finalize_stats(c, lps, 1, push, &c->stats_seq)) != HALOS_OK) return rc;
+    c->stats_seq += 1;
     apply_commit(c, lps, worker, push);
     if (push_due) *push_due = due ? 1 : 0;
     return HALOS_OK;
@@ -435,6 +470,9 @@ int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool pu
     a.acc = s.acc;
     a.anchor = s.anchor;
     a.outbox = s.outbox;
+    a.partial_delta = c->d_partial_delta;
+    a.partial_theta = c->d_partial_theta;
+    a.partial_Delta = c->d_partial_Delta;
     a.eps = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.inv_n = 1.0f / (float)c->cfg.delay_l;
@@ -443,12 +481,15 @@ int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool pu
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     const bool any = a.refresh_mask != 0;
     Timer tm(c, HALOS_K_ARRIVE_MULTI);
-    if (any) {
-        if (push) arrive_multi_dn_kernel<W, NB, true, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_multi_dn_kernel<W, NB, true, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+    const Chunk* table = next_table(c);
+    if (stats_on(c)) {
+#define CALL(A, P) arrive_multi_dn_kernel<W, NB, A, P, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(table, a)
+        HALOS_PICK2(any, push, CALL);
+#undef CALL
     } else {
-        if (push) arrive_multi_dn_kernel<W, NB, false, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
-        else arrive_multi_dn_kernel<W, NB, false, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+#define CALL(A, P) arrive_multi_dn_kernel<W, NB, A, P, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(table, a)
+        HALOS_PICK2(any, push, CALL);
+#undef CALL
     }
     tm.stop();
     c->launches++;
@@ -474,14 +515,19 @@ int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push)
     a.ml = s.ml;
     a.anchor = s.anchor;
     a.outbox = s.outbox;
+    a.partial_delta = c->d_partial_delta;
+    a.partial_theta = c->d_partial_theta;
+    a.partial_Delta = c->d_partial_Delta;
     a.eta = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.omb = 1.0f - c->cfg.beta_l;
     constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     Timer tm(c, HALOS_K_ARRIVE_MULTI);
-    if (push) arrive_multi_kernel<W, NB, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
-    else arrive_multi_kernel<W, NB, false, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(next_table(c), a);
+    const Chunk* table = next_table(c);
+#define CALL(P, S) arrive_multi_kernel<W, NB, P, S, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(table, a)
+    HALOS_PICK2(push, stats_on(c), CALL);
+#undef CALL
     tm.stop();
     c->launches++;
     c->batched_arrivals += NB;
@@ -506,6 +552,11 @@ int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool 
         case 7: rc = launch_arrive_multi<W, 7>(c, s, q.data(), push); break;
         case 8: rc = launch_arrive_multi<W, 8>(c, s, q.data(), push); break;
         default: rc = fail(c, HALOS_ERR_INVALID_ARG, "internal: batch larger than %d", kMaxBatch);
+    }
+    if (rc == HALOS_OK && stats_on(c)) {
+        uint64_t seq[kMaxBatch];
+        for (size_t j = 0; j < q.size(); ++j) seq[j] = q[j].seq;
+        rc = finalize_stats(c, lps, (uint32_t)q.size(), push, seq);
     }
     q.clear();
     return rc;
@@ -584,16 +635,15 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
         return fail(nullptr, HALOS_ERR_INVALID_ARG, "unknown optimizer");
     if (cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV && (cfg->delay_l == 0 || cfg->delay_g == 0))
         return fail(nullptr, HALOS_ERR_INVALID_ARG, "delays must be at least 1");
-    if (cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV && (cfg->flags & HALOS_FLAG_STATS))
-        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "statistics are not available with the delayed Nesterov optimizer");
-    if ((cfg->flags & HALOS_FLAG_MATERIALISE_DELTA) &&
-        ((cfg->flags & HALOS_FLAG_STATS) || cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV))
-        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "materialised deltas combine neither with statistics nor with delayed Nesterov");
+    if ((cfg->flags & HALOS_FLAG_MATERIALISE_DELTA) && cfg->optimizer == HALOS_OPT_DELAYED_NESTEROV)
+        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "materialised deltas do not combine with delayed Nesterov");
     if ((cfg->alloc == nullptr) != (cfg->free_ == nullptr)) return fail(nullptr, HALOS_ERR_INVALID_ARG, "alloc and free_ go together");
     for (uint32_t w = 0; w < cfg->n_workers; ++w)
         if (cfg->worker_lps[w] >= cfg->n_lps) return fail(nullptr, HALOS_ERR_INVALID_ARG, "worker_lps[%u] out of range", w);
     uint32_t chunk_elems = cfg->chunk_elems ? cfg->chunk_elems : kDefaultChunkElems;
     if (chunk_elems % 8 != 0) return fail(nullptr, HALOS_ERR_INVALID_ARG, "chunk_elems must be a positive multiple of 8");
+    if ((cfg->flags & HALOS_FLAG_STATS) && chunk_elems > kStatMaxChunk)
+        return fail(nullptr, HALOS_ERR_UNSUPPORTED, "statistics need chunk_elems <= %u", kStatMaxChunk);
 
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
@@ -656,9 +706,9 @@ int halos_create(const halos_config* cfg, const float* theta_init_dev, halos_ctx
     ok &= (c->d_tensor_chunk_begin = (uint32_t*)A((nt + 1) * 4)) != nullptr;
     ok &= (c->d_ptr_tables = (const void**)A((size_t)cfg->n_workers * nt * 8)) != nullptr;
     if (cfg->flags & HALOS_FLAG_STATS) {
-        ok &= (c->d_partial_delta = (double*)A(nc * 8)) != nullptr;
+        ok &= (c->d_partial_delta = (double*)A((size_t)kMaxBatch * nc * 8)) != nullptr;   // [arrival of a launch][chunk]
         ok &= (c->d_partial_Delta = (double*)A(nc * 8)) != nullptr;
-        ok &= (c->d_partial_theta = (double*)A(nc * 8)) != nullptr;
+        ok &= (c->d_partial_theta = (double*)A((size_t)kMaxBatch * nc * 8)) != nullptr;
         ok &= (c->d_stats = (double*)A((size_t)3 * cfg->n_lps * nt * 8)) != nullptr;
     }
     ok &= (c->Theta = (float*)S(P * 4)) != nullptr;
@@ -749,6 +799,17 @@ int halos_worker_delta(halos_ctx* c, uint32_t worker, const void* flat, const vo
     {
         int rq = flush_worker(c, worker);   // a still-queued arrival of this worker reads its old result / table
         if (rq != HALOS_OK) return rq;
+    }
+    if (stats_on(c)) {
+        // which tensors of this result can take the vector path (their first full chunk starts `head` elements in)
+        const size_t ntens = c->tensor_numel.size();
+        w.vec_aligned.assign(ntens, 0);
+        for (size_t k = 0; k < ntens; ++k) {
+            const uint64_t head = (kVE - (c->tensor_off[k] % kVE)) % kVE;
+            const uintptr_t first = flat ? reinterpret_cast<uintptr_t>(flat) + (c->tensor_off[k] + head) * c->wb
+                                         : reinterpret_cast<uintptr_t>(ptrs[k]) + head * c->wb;
+            w.vec_aligned[k] = (first % (kVE * c->wb)) == 0;
+        }
     }
     if (flat) {
         if (reinterpret_cast<uintptr_t>(flat) % c->wb) return fail(c, HALOS_ERR_INVALID_ARG, "thetaH not aligned to its element size");
@@ -856,8 +917,11 @@ int halos_lps_push(halos_ctx* c, uint32_t lps) {
     c->launches++;
     CU(c, cudaGetLastError());
     if (stats) {
-        int rc = finalize_stats(c, 1, lps);
-        if (rc != HALOS_OK) return rc;
+        const uint32_t nt = (uint32_t)c->tensor_numel.size();
+        stats_finalize_push_kernel<<<nt, 32, 0, c->stream>>>(c->d_partial_Delta, c->d_tensor_chunk_begin,
+                                                             c->d_stats + ((size_t)1 * c->cfg.n_lps + lps) * nt, nt);
+        c->launches++;
+        CU(c, cudaGetLastError());
     }
     s.phase = HALOS_PUSHED;
     s.t_push = s.t;
@@ -917,6 +981,51 @@ static int pull_impl(halos_ctx* c, uint32_t lps) {
     return HALOS_OK;
 }
 
+// GPS update for this LPS's Delta and the merge of the answer into the same LPS as one launch.  The caller has
+// launched whatever was queued for this LPS.
+static int gps_pull_impl(halos_ctx* c, uint32_t lps) {
+    if (lps >= c->cfg.n_lps) return fail(c, HALOS_ERR_INVALID_ARG, "lps out of range");
+    LpsState& s = c->lps[lps];
+    if (s.phase != HALOS_PUSHED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Delta in flight", lps);
+    CU(c, cudaSetDevice(c->cfg.device));
+    GpsPullArgs a;
+    a.outbox = s.outbox;
+    a.Theta = c->Theta;
+    a.Mg = c->Mg;
+    a.acc = c->acc_g;
+    a.inbox = s.inbox;
+    a.th = s.th;
+    a.anchor = s.anchor;
+    a.eta = c->cfg.eta_g;
+    a.beta = c->cfg.beta_g;
+    a.omb = 1.0f - c->cfg.beta_g;
+    a.inv_n = 1.0f / (float)(c->cfg.delay_g ? c->cfg.delay_g : 1);
+    a.eps_n = c->cfg.eta_g * a.inv_n;
+    a.alpha = c->cfg.alpha;
+    a.oma = 1.0f - c->cfg.alpha;
+    const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
+    Timer tm(c, HALOS_K_GPS_PULL);
+    const Chunk* table = next_table(c);
+    if (c->cfg.optimizer != HALOS_OPT_DELAYED_NESTEROV) gps_pull_kernel<0, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a);
+    else if (((c->gps_iter + 1) % c->cfg.delay_g) == 0) gps_pull_kernel<2, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a);
+    else gps_pull_kernel<1, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a);
+    tm.stop();
+    c->launches++;
+    CU(c, cudaGetLastError());
+    c->gps_iter += 1;
+    s.inbox_iter = c->gps_iter;
+    s.t_last = s.t;
+    s.phase = HALOS_IDLE;
+    return HALOS_OK;
+}
+
+int halos_gps_merge_pull(halos_ctx* c, uint32_t lps) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    int rq = flush_all(c);
+    if (rq != HALOS_OK) return rq;
+    return gps_pull_impl(c, lps);
+}
+
 // ------------------------------------------------------------------------------ event-queue driver
 // Events are taken in trace order: counters, phases, the log and the producer calls follow that order
 // exactly.  With max_batch > 1 the LAUNCH of an arrival may be deferred: arrivals at one LPS wait in
@@ -932,7 +1041,6 @@ int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_p
     if (n && !ev) return fail(c, HALOS_ERR_INVALID_ARG, "null event array");
     if (max_batch == 0) max_batch = 1;
     if (max_batch > (uint32_t)kMaxBatch) max_batch = kMaxBatch;
-    if (c->cfg.flags & HALOS_FLAG_STATS) max_batch = 1;   // per-arrival statistics need per-arrival launches
     const bool immediate = (c->cfg.flags & HALOS_FLAG_MATERIALISE_DELTA) != 0;   // launched event by event
     std::vector<std::vector<Deferred>>& queue = c->deferred;
     int rc = HALOS_OK;
@@ -976,16 +1084,47 @@ int halos_replay_stream(halos_ctx* c, const halos_event* ev, uint32_t n, halos_p
                     } else {
                         const bool refresh = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV &&
                                              ((c->lps[e.lps].t + 1) % c->cfg.delay_l) == 0;
-                        q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr, refresh});
-                        rec.fused = (uint8_t)(q.size() > 1 || push);
-                        apply_commit(c, e.lps, e.worker, push);
-                        if (push || q.size() >= max_batch) rc = flush_deferred(c, e.lps, q, push);
+                        // statistics are reduced per vector or per element depending on the alignment of the
+                        // caller's tensors; only arrivals that agree on it tensor by tensor share a launch, so that
+                        // a fused launch reports the sums of the single launches bit for bit
+                        if (stats_on(c) && !q.empty() && c->workers[q[0].worker].vec_aligned != w.vec_aligned)
+                            rc = flush_deferred(c, e.lps, q, false);
+                        if (rc == HALOS_OK) {
+                            q.push_back(Deferred{e.worker, w.pending == PEND_FLAT ? w.flat : nullptr, refresh, c->stats_seq++});
+                            rec.fused = (uint8_t)(q.size() > 1 || push);
+                            apply_commit(c, e.lps, e.worker, push);
+                            if (push || q.size() >= max_batch) rc = flush_deferred(c, e.lps, q, push);
+                        }
                     }
                     rec.pushed = (uint8_t)push;
                 }
             }
         } else if (e.kind == HALOS_EV_GPS_RECV) {
-            rc = halos_gps_merge(c, e.lps);
+            // GPS_RECV(l) directly followed by PULL(l): one fused launch (only with multi-event fusion enabled)
+            if (max_batch > 1 && k + 1 < n && ev[k + 1].kind == HALOS_EV_PULL && ev[k + 1].lps == e.lps &&
+                c->lps[e.lps].phase == HALOS_PUSHED) {
+                rc = flush_deferred(c, e.lps, queue[e.lps], false);   // arrivals before the PULL come first
+                const uint64_t t_last_before = c->lps[e.lps].t_last;
+                if (rc == HALOS_OK) rc = gps_pull_impl(c, e.lps);
+                if (rc == HALOS_OK) {
+                    rec.fused = 1;
+                    if (log) {
+                        rec.t = c->lps[e.lps].t;
+                        rec.t_last = t_last_before;
+                        rec.gps_iter = c->gps_iter;
+                        log[k] = rec;
+                    }
+                    ++k;                                              // the PULL is done as well
+                    std::memset(&rec, 0, sizeof rec);
+                    rec.index = k;
+                    rec.kind = HALOS_EV_PULL;
+                    rec.lps = e.lps;
+                    rec.fused = 1;
+                    rec.gps_lag = 0;                                  // it merges the Theta_i this very iteration produced
+                }
+            } else {
+                rc = halos_gps_merge(c, e.lps);
+            }
         } else if (e.kind == HALOS_EV_PULL) {
             rc = flush_deferred(c, e.lps, queue[e.lps], false);
             if (rc == HALOS_OK) {
@@ -1236,6 +1375,19 @@ int halos_stats(halos_ctx* c, uint32_t what, uint32_t lps, double* out) {
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaMemcpyAsync(out, c->d_stats + ((size_t)what * c->cfg.n_lps + lps) * nt, nt * 8, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
+    return HALOS_OK;
+}
+
+int halos_stats_log(halos_ctx* c, double* log_dev, uint64_t capacity_records) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (!stats_on(c)) return fail(c, HALOS_ERR_BAD_STATE, "context was created without HALOS_FLAG_STATS");
+    if ((log_dev == nullptr) != (capacity_records == 0)) return fail(c, HALOS_ERR_INVALID_ARG, "log pointer and capacity go together");
+    if (reinterpret_cast<uintptr_t>(log_dev) & 7) return fail(c, HALOS_ERR_INVALID_ARG, "log not aligned to 8 bytes");
+    int rq = flush_all(c);   // queued arrivals belong to the previous log
+    if (rq != HALOS_OK) return rq;
+    c->stats_log = log_dev;
+    c->stats_log_capacity = capacity_records;
+    c->stats_seq = 0;
     return HALOS_OK;
 }
 

@@ -209,20 +209,36 @@ template <> struct WTraits<uint16_t> {
     static __device__ __forceinline__ void store1(uint16_t* p, float v) { *p = (uint16_t)bf16_narrow(v); }
 };
 
-// ---------------------------------------------------------------- block reduction (statistics only)
-// Deterministic: fixed shuffle tree inside a warp, then warp 0 adds the warp sums in order.
-__device__ __forceinline__ double block_sum(double v, double* smem /* kThreads/32 doubles */) {
+// ---------------------------------------------------------------- statistics reduction
+// Squared norms are reduced in a canonical order that does not depend on the CTA size or on how many
+// arrivals a launch fuses, so that a fused launch reports the same fp64 sums, bit for bit, as the
+// launches it replaces:
+//   item     one vector of VE consecutive elements (vector path) or one element (scalar path); its value is
+//            the fp32 sum of squares accumulated with fmaf from 0 in element order;
+//   row      32 consecutive items of a chunk, summed in fp64 by a fixed shuffle tree (absent items count 0);
+//   chunk    row sums added in fp64 in increasing row order (vector rows first, then scalar rows).
+// A chunk of up to kStatMaxChunk elements has at most kStatRows rows.
+constexpr int kStatRows = 256;
+constexpr uint32_t kStatMaxChunk = kStatRows * 32;
+
+__device__ __forceinline__ double row_sum(float item) {   // every lane of the warp calls it; valid in lane 0
+    double v = (double)item;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) smem[warp] = v;
-    __syncthreads();
-    double total = 0.0;
-    if (threadIdx.x == 0) {
+    return v;
+}
+template <int VE>
+__device__ __forceinline__ float sumsq(const FVec<VE>& d) {
+    float acc = 0.f;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) total += smem[w];
-    }
-    return total;  // valid in thread 0
+    for (int e = 0; e < VE; ++e) acc = fmaf(d.v[e], d.v[e], acc);
+    return acc;
+}
+// Adds the rows of quantity q in order; called by thread q (q < number of quantities) after a __syncthreads().
+__device__ __forceinline__ double rows_total(const double* rows, uint32_t nrows) {
+    double t = 0.0;
+    for (uint32_t r = 0; r < nrows; ++r) t += rows[r];
+    return t;
 }
 
 // =====================================================================================================
@@ -244,13 +260,6 @@ struct ArriveArgs {
     float eta, beta, omb;
 };
 
-template <int VE>
-__device__ __forceinline__ float sumsq(const FVec<VE>& d, float acc) {
-#pragma unroll
-    for (int e = 0; e < VE; ++e) acc = fmaf(d.v[e], d.v[e], acc);
-    return acc;
-}
-
 template <class W, bool PUSH, bool STATS, int UNROLL, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
@@ -263,7 +272,9 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
     const float* an = PUSH ? a.anchor + c.begin : nullptr;
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eta = a.eta, beta = a.beta, omb = a.omb;
-    float acc_d = 0.f, acc_D = 0.f, acc_x = 0.f;
+    __shared__ double srow[STATS ? 3 : 1][STATS ? kStatRows : 1];   // [delta^2, theta^2, Delta^2][row]
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;   // rows of the vector path
 
     // vector path: the chunk starts on a VE-element boundary of the packed state (bases are 256-byte
     // aligned) and the caller's theta_H pointer is aligned to one vector of its own type
@@ -271,6 +282,7 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
     uint32_t done = 0;
     if (vec_ok) {
         const uint32_t nvec = c.count / VE;
+        nrv = (nvec + 31u) >> 5;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
             FVec<VE> vh[UNROLL], vs[UNROLL], vx[UNROLL], vm[UNROLL], va[UNROLL];
 #pragma unroll
@@ -288,6 +300,7 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
+                float q_d = 0.f, q_x = 0.f, q_D = 0.f;
                 if (v < nvec) {
                     const size_t o = (size_t)VE * v;
                     FVec<VE> d;
@@ -300,15 +313,26 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
                     stf<VE, STREAM>(ml + o, vm[u]);
                     T::template store<VE, STREAM>(s0 + o, vx[u]);
                     if (STATS) {
-                        acc_d = sumsq<VE>(d, acc_d);
-                        acc_x = sumsq<VE>(vx[u], acc_x);
+                        q_d = sumsq<VE>(d);
+                        q_x = sumsq<VE>(vx[u]);
                     }
                     if (PUSH) {
                         FVec<VE> D;
 #pragma unroll
                         for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx[u].v[e], va[u].v[e]);
                         stf<VE, STREAM>(ob + o, D);
-                        if (STATS) acc_D = sumsq<VE>(D, acc_D);
+                        if (STATS) q_D = sumsq<VE>(D);
+                    }
+                }
+                if (STATS) {
+                    const uint32_t vb = base + u * kThreads + warp32;   // first item of this warp's row
+                    if (vb < nvec) {
+                        const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+                        if (lane == 0) {
+                            srow[0][vb >> 5] = r_d;
+                            srow[1][vb >> 5] = r_x;
+                            if (PUSH) srow[2][vb >> 5] = r_D;
+                        }
                     }
                 }
             }
@@ -316,34 +340,42 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
         done = nvec * VE;
     }
     // ragged tail (or a whole chunk whose pointers do not share the vector alignment): scalar
-    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
-        float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
-        float x = th[j], m = ml[j];
-        model_update(x, m, d, eta, beta, omb);
-        th[j] = x;
-        ml[j] = m;
-        T::store1(s0 + j, x);
-        if (STATS) {
-            acc_d = fmaf(d, d, acc_d);
-            acc_x = fmaf(x, x, acc_x);
+    for (uint32_t jb = done + warp32; jb < c.count; jb += kThreads) {
+        const uint32_t j = jb + lane;
+        float q_d = 0.f, q_x = 0.f, q_D = 0.f;
+        if (j < c.count) {
+            float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
+            float x = th[j], m = ml[j];
+            model_update(x, m, d, eta, beta, omb);
+            th[j] = x;
+            ml[j] = m;
+            T::store1(s0 + j, x);
+            if (STATS) {
+                q_d = fmaf(d, d, 0.f);
+                q_x = fmaf(x, x, 0.f);
+            }
+            if (PUSH) {
+                float D = __fsub_rn(x, an[j]);
+                ob[j] = D;
+                if (STATS) q_D = fmaf(D, D, 0.f);
+            }
         }
-        if (PUSH) {
-            float D = __fsub_rn(x, an[j]);
-            ob[j] = D;
-            if (STATS) acc_D = fmaf(D, D, acc_D);
+        if (STATS) {
+            const uint32_t row = nrv + ((jb - done) >> 5);
+            const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+            if (lane == 0) {
+                srow[0][row] = r_d;
+                srow[1][row] = r_x;
+                if (PUSH) srow[2][row] = r_D;
+            }
         }
     }
     if (STATS) {
-        __shared__ double red[kThreads / 32];
-        double t = block_sum((double)acc_d, red);
-        if (threadIdx.x == 0) a.partial_delta[blockIdx.x] = t;
         __syncthreads();
-        double t3 = block_sum((double)acc_x, red);
-        if (threadIdx.x == 0) a.partial_theta[blockIdx.x] = t3;
-        if (PUSH) {
-            __syncthreads();
-            double t2 = block_sum((double)acc_D, red);
-            if (threadIdx.x == 0) a.partial_Delta[blockIdx.x] = t2;
+        const uint32_t nrows = nrv + ((c.count - done + 31u) >> 5);
+        if (threadIdx.x < (PUSH ? 3u : 2u)) {
+            double* dst = threadIdx.x == 0 ? a.partial_delta : threadIdx.x == 1 ? a.partial_theta : a.partial_Delta;
+            dst[blockIdx.x] = rows_total(srow[threadIdx.x], nrows);
         }
     }
 }
@@ -369,10 +401,42 @@ struct ArriveMultiArgs {
     float* ml;
     const float* anchor;
     float* outbox;
+    double* partial_delta;               // [NB][n_chunks] sum delta^2 of arrival j per chunk   (STATS only)
+    double* partial_theta;               // [NB][n_chunks] sum theta^2 right after arrival j    (STATS only)
+    double* partial_Delta;               // [n_chunks]     sum Delta^2                          (STATS && PUSH)
     float eta, beta, omb;
 };
 
-template <class W, int NB, bool PUSH, bool STREAM, int VE, int TPB>
+// Statistics of a fused launch: quantity 2j = delta^2 of arrival j, 2j+1 = theta^2 after arrival j, 2 NB = Delta^2.
+template <int NB, bool PUSH>
+__device__ __forceinline__ void multi_stats_rows(double (*srow)[kStatRows + 1], uint32_t row, uint32_t lane,
+                                                 const float* q_d, const float* q_x, float q_D) {
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        const double r_d = row_sum(q_d[j]), r_x = row_sum(q_x[j]);
+        if (lane == 0) {
+            srow[2 * j][row] = r_d;
+            srow[2 * j + 1][row] = r_x;
+        }
+    }
+    if (PUSH) {
+        const double r_D = row_sum(q_D);
+        if (lane == 0) srow[2 * NB][row] = r_D;
+    }
+}
+template <int NB, bool PUSH>
+__device__ __forceinline__ void multi_stats_finish(double (*srow)[kStatRows + 1], uint32_t nrows, double* partial_delta,
+                                                   double* partial_theta, double* partial_Delta) {
+    __syncthreads();
+    const uint32_t q = threadIdx.x;
+    if (q < 2u * NB + (PUSH ? 1u : 0u)) {
+        const double t = rows_total(srow[q], nrows);
+        if (q == 2u * NB) partial_Delta[blockIdx.x] = t;
+        else ((q & 1u) ? partial_theta : partial_delta)[(size_t)(q >> 1) * gridDim.x + blockIdx.x] = t;
+    }
+}
+
+template <class W, int NB, bool PUSH, bool STATS, bool STREAM, int VE, int TPB>
 __global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
 arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
     using T = WTraits<W>;
@@ -391,52 +455,86 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
     const float* an = PUSH ? a.anchor + c.begin : nullptr;
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eta = a.eta, beta = a.beta, omb = a.omb;
+    __shared__ double srow[STATS ? 2 * NB + 1 : 1][STATS ? kStatRows + 1 : 1];
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;
     uint32_t done = 0;
     if (vec_ok) {
         const uint32_t nvec = c.count / VE;
-        for (uint32_t v = threadIdx.x; v < nvec; v += TPB) {
-            const size_t o = (size_t)VE * v;
-            FVec<VE> vh[NB], vs[NB], vx, vm, va;
+        nrv = (nvec + 31u) >> 5;
+        for (uint32_t vb = warp32; vb < nvec; vb += TPB) {   // a warp walks its rows of 32 vectors together
+            const uint32_t v = vb + lane;
+            float q_d[NB], q_x[NB], q_D = 0.f;
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                vh[j] = T::template load<VE, STREAM>(h[j] + o);
-                vs[j] = T::template load<VE, STREAM>(s0[j] + o);
-            }
-            vx = ldf<VE, STREAM>(th + o);
-            vm = ldf<VE, STREAM>(ml + o);
-            if (PUSH) va = ldf<VE, STREAM>(an + o);
+            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            if (v < nvec) {
+                const size_t o = (size_t)VE * v;
+                FVec<VE> vh[NB], vs[NB], vx, vm, va;
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-#pragma unroll
-                for (int e = 0; e < VE; ++e) {
-                    const float d = __fsub_rn(vh[j].v[e], vs[j].v[e]);
-                    model_update(vx.v[e], vm.v[e], d, eta, beta, omb);
+                for (int j = 0; j < NB; ++j) {
+                    vh[j] = T::template load<VE, STREAM>(h[j] + o);
+                    vs[j] = T::template load<VE, STREAM>(s0[j] + o);
                 }
-                T::template store<VE, STREAM>(s0[j] + o, vx);   // worker j restarts from the model after ITS update
-            }
-            stf<VE, STREAM>(th + o, vx);
-            stf<VE, STREAM>(ml + o, vm);
-            if (PUSH) {
-                FVec<VE> D;
+                vx = ldf<VE, STREAM>(th + o);
+                vm = ldf<VE, STREAM>(ml + o);
+                if (PUSH) va = ldf<VE, STREAM>(an + o);
 #pragma unroll
-                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
-                stf<VE, STREAM>(ob + o, D);
+                for (int j = 0; j < NB; ++j) {
+                    FVec<VE> d;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) {
+                        d.v[e] = __fsub_rn(vh[j].v[e], vs[j].v[e]);
+                        model_update(vx.v[e], vm.v[e], d.v[e], eta, beta, omb);
+                    }
+                    T::template store<VE, STREAM>(s0[j] + o, vx);   // worker j restarts from the model after ITS update
+                    if (STATS) {
+                        q_d[j] = sumsq<VE>(d);
+                        q_x[j] = sumsq<VE>(vx);
+                    }
+                }
+                stf<VE, STREAM>(th + o, vx);
+                stf<VE, STREAM>(ml + o, vm);
+                if (PUSH) {
+                    FVec<VE> D;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                    stf<VE, STREAM>(ob + o, D);
+                    if (STATS) q_D = sumsq<VE>(D);
+                }
             }
+            if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, vb >> 5, lane, q_d, q_x, q_D);
         }
         done = nvec * VE;
     }
-    for (uint32_t i = done + threadIdx.x; i < c.count; i += TPB) {
-        float x = th[i], m = ml[i];
+    for (uint32_t ib = done + warp32; ib < c.count; ib += TPB) {
+        const uint32_t i = ib + lane;
+        float q_d[NB], q_x[NB], q_D = 0.f;
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
-            const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
-            model_update(x, m, d, eta, beta, omb);
-            T::store1(s0[j] + i, x);
+        for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+        if (i < c.count) {
+            float x = th[i], m = ml[i];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
+                model_update(x, m, d, eta, beta, omb);
+                T::store1(s0[j] + i, x);
+                if (STATS) {
+                    q_d[j] = fmaf(d, d, 0.f);
+                    q_x[j] = fmaf(x, x, 0.f);
+                }
+            }
+            th[i] = x;
+            ml[i] = m;
+            if (PUSH) {
+                const float D = __fsub_rn(x, an[i]);
+                ob[i] = D;
+                if (STATS) q_D = fmaf(D, D, 0.f);
+            }
         }
-        th[i] = x;
-        ml[i] = m;
-        if (PUSH) ob[i] = __fsub_rn(x, an[i]);
+        if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, nrv + ((ib - done) >> 5), lane, q_d, q_x, q_D);
     }
+    if constexpr (STATS)
+        multi_stats_finish<NB, PUSH>(srow, nrv + ((c.count - done + 31u) >> 5), a.partial_delta, a.partial_theta, a.partial_Delta);
 }
 
 // =====================================================================================================
@@ -455,10 +553,13 @@ struct ArriveDnArgs {
     float* acc;
     const float* anchor;
     float* outbox;
+    double* partial_delta;   // statistics, as in ArriveArgs
+    double* partial_Delta;
+    double* partial_theta;
     float eps, beta, inv_n, eps_n;
 };
 
-template <class W, bool REFRESH, bool PUSH, bool STREAM, int VE>
+template <class W, bool REFRESH, bool PUSH, bool STATS, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 arrive_dn_kernel(const Chunk* __restrict__ chunks, ArriveDnArgs<W> a) {
     using T = WTraits<W>;
@@ -471,48 +572,98 @@ arrive_dn_kernel(const Chunk* __restrict__ chunks, ArriveDnArgs<W> a) {
     const float* an = PUSH ? a.anchor + c.begin : nullptr;
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eps = a.eps, beta = a.beta, inv_n = a.inv_n, eps_n = a.eps_n;
+    __shared__ double srow[STATS ? 3 : 1][STATS ? kStatRows : 1];
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;
     const bool vec_ok = ((c.begin % VE) == 0) && ((reinterpret_cast<uintptr_t>(h) % (VE * sizeof(W))) == 0);
     uint32_t done = 0;
     if (vec_ok) {
         const uint32_t nvec = c.count / VE;
-        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
-            const size_t o = (size_t)VE * v;
-            FVec<VE> vh = T::template load<VE, STREAM>(h + o);
-            FVec<VE> vs = T::template load<VE, STREAM>(s0 + o);
-            FVec<VE> vx = ldf<VE, STREAM>(th + o);
-            FVec<VE> vc = ldf<VE, STREAM>(ac + o);
-            FVec<VE> vm, va;
-            if (REFRESH) vm = ldf<VE, STREAM>(ml + o);
-            if (PUSH) va = ldf<VE, STREAM>(an + o);
+        nrv = (nvec + 31u) >> 5;
+        for (uint32_t vb = warp32; vb < nvec; vb += kThreads) {
+            const uint32_t v = vb + lane;
+            float q_d = 0.f, q_x = 0.f, q_D = 0.f;
+            if (v < nvec) {
+                const size_t o = (size_t)VE * v;
+                FVec<VE> vh = T::template load<VE, STREAM>(h + o);
+                FVec<VE> vs = T::template load<VE, STREAM>(s0 + o);
+                FVec<VE> vx = ldf<VE, STREAM>(th + o);
+                FVec<VE> vc = ldf<VE, STREAM>(ac + o);
+                FVec<VE> vm, va, d;
+                if (REFRESH) vm = ldf<VE, STREAM>(ml + o);
+                if (PUSH) va = ldf<VE, STREAM>(an + o);
 #pragma unroll
-            for (int e = 0; e < VE; ++e) {
-                const float d = __fsub_rn(vh.v[e], vs.v[e]);
-                float m = REFRESH ? vm.v[e] : 0.f;
-                delayed_nesterov<REFRESH>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
-                if (REFRESH) vm.v[e] = m;
+                for (int e = 0; e < VE; ++e) {
+                    d.v[e] = __fsub_rn(vh.v[e], vs.v[e]);
+                    float m = REFRESH ? vm.v[e] : 0.f;
+                    delayed_nesterov<REFRESH>(vx.v[e], m, vc.v[e], d.v[e], eps, beta, inv_n, eps_n);
+                    if (REFRESH) vm.v[e] = m;
+                }
+                stf<VE, STREAM>(th + o, vx);
+                stf<VE, STREAM>(ac + o, vc);
+                if (REFRESH) stf<VE, STREAM>(ml + o, vm);
+                T::template store<VE, STREAM>(s0 + o, vx);
+                if (STATS) {
+                    q_d = sumsq<VE>(d);
+                    q_x = sumsq<VE>(vx);
+                }
+                if (PUSH) {
+                    FVec<VE> D;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                    stf<VE, STREAM>(ob + o, D);
+                    if (STATS) q_D = sumsq<VE>(D);
+                }
             }
-            stf<VE, STREAM>(th + o, vx);
-            stf<VE, STREAM>(ac + o, vc);
-            if (REFRESH) stf<VE, STREAM>(ml + o, vm);
-            T::template store<VE, STREAM>(s0 + o, vx);
-            if (PUSH) {
-                FVec<VE> D;
-#pragma unroll
-                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
-                stf<VE, STREAM>(ob + o, D);
+            if (STATS) {
+                const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+                if (lane == 0) {
+                    srow[0][vb >> 5] = r_d;
+                    srow[1][vb >> 5] = r_x;
+                    if (PUSH) srow[2][vb >> 5] = r_D;
+                }
             }
         }
         done = nvec * VE;
     }
-    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
-        const float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
-        float x = th[j], acc = ac[j], m = REFRESH ? ml[j] : 0.f;
-        delayed_nesterov<REFRESH>(x, m, acc, d, eps, beta, inv_n, eps_n);
-        th[j] = x;
-        ac[j] = acc;
-        if (REFRESH) ml[j] = m;
-        T::store1(s0 + j, x);
-        if (PUSH) ob[j] = __fsub_rn(x, an[j]);
+    for (uint32_t jb = done + warp32; jb < c.count; jb += kThreads) {
+        const uint32_t j = jb + lane;
+        float q_d = 0.f, q_x = 0.f, q_D = 0.f;
+        if (j < c.count) {
+            const float d = __fsub_rn(T::load1(h + j), T::load1(s0 + j));
+            float x = th[j], acc = ac[j], m = REFRESH ? ml[j] : 0.f;
+            delayed_nesterov<REFRESH>(x, m, acc, d, eps, beta, inv_n, eps_n);
+            th[j] = x;
+            ac[j] = acc;
+            if (REFRESH) ml[j] = m;
+            T::store1(s0 + j, x);
+            if (STATS) {
+                q_d = fmaf(d, d, 0.f);
+                q_x = fmaf(x, x, 0.f);
+            }
+            if (PUSH) {
+                const float D = __fsub_rn(x, an[j]);
+                ob[j] = D;
+                if (STATS) q_D = fmaf(D, D, 0.f);
+            }
+        }
+        if (STATS) {
+            const uint32_t row = nrv + ((jb - done) >> 5);
+            const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+            if (lane == 0) {
+                srow[0][row] = r_d;
+                srow[1][row] = r_x;
+                if (PUSH) srow[2][row] = r_D;
+            }
+        }
+    }
+    if (STATS) {
+        __syncthreads();
+        const uint32_t nrows = nrv + ((c.count - done + 31u) >> 5);
+        if (threadIdx.x < (PUSH ? 3u : 2u)) {
+            double* dst = threadIdx.x == 0 ? a.partial_delta : threadIdx.x == 1 ? a.partial_theta : a.partial_Delta;
+            dst[blockIdx.x] = rows_total(srow[threadIdx.x], nrows);
+        }
     }
 }
 
@@ -583,11 +734,14 @@ struct ArriveMultiDnArgs {
     float* acc;
     const float* anchor;
     float* outbox;
+    double* partial_delta;   // statistics, as in ArriveMultiArgs
+    double* partial_theta;
+    double* partial_Delta;
     float eps, beta, inv_n, eps_n;
     uint32_t refresh_mask;
 };
 
-template <class W, int NB, bool ANYREF, bool PUSH, bool STREAM, int VE, int TPB>
+template <class W, int NB, bool ANYREF, bool PUSH, bool STATS, bool STREAM, int VE, int TPB>
 __global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
 arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a) {
     using T = WTraits<W>;
@@ -608,67 +762,101 @@ arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a)
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eps = a.eps, beta = a.beta, inv_n = a.inv_n, eps_n = a.eps_n;
     const uint32_t mask = a.refresh_mask;
+    __shared__ double srow[STATS ? 2 * NB + 1 : 1][STATS ? kStatRows + 1 : 1];
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;
     uint32_t done = 0;
     if (vec_ok) {
         const uint32_t nvec = c.count / VE;
-        for (uint32_t v = threadIdx.x; v < nvec; v += TPB) {
-            const size_t o = (size_t)VE * v;
-            FVec<VE> vh[NB], vs[NB], vx, vc, vm, va;
+        nrv = (nvec + 31u) >> 5;
+        for (uint32_t vb = warp32; vb < nvec; vb += TPB) {
+            const uint32_t v = vb + lane;
+            float q_d[NB], q_x[NB], q_D = 0.f;
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                vh[j] = T::template load<VE, STREAM>(h[j] + o);
-                vs[j] = T::template load<VE, STREAM>(s0[j] + o);
-            }
-            vx = ldf<VE, STREAM>(th + o);
-            vc = ldf<VE, STREAM>(ac + o);
-            if (ANYREF) vm = ldf<VE, STREAM>(ml + o);
-            if (PUSH) va = ldf<VE, STREAM>(an + o);
+            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            if (v < nvec) {
+                const size_t o = (size_t)VE * v;
+                FVec<VE> vh[NB], vs[NB], vx, vc, vm, va;
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                const bool refresh = ANYREF && ((mask >> j) & 1u);   // uniform over the grid
+                for (int j = 0; j < NB; ++j) {
+                    vh[j] = T::template load<VE, STREAM>(h[j] + o);
+                    vs[j] = T::template load<VE, STREAM>(s0[j] + o);
+                }
+                vx = ldf<VE, STREAM>(th + o);
+                vc = ldf<VE, STREAM>(ac + o);
+                if (ANYREF) vm = ldf<VE, STREAM>(ml + o);
+                if (PUSH) va = ldf<VE, STREAM>(an + o);
 #pragma unroll
-                for (int e = 0; e < VE; ++e) {
-                    const float d = __fsub_rn(vh[j].v[e], vs[j].v[e]);
-                    if (refresh) {
-                        float m = vm.v[e];
-                        delayed_nesterov<true>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
-                        vm.v[e] = m;
-                    } else {
-                        float m = 0.f;
-                        delayed_nesterov<false>(vx.v[e], m, vc.v[e], d, eps, beta, inv_n, eps_n);
+                for (int j = 0; j < NB; ++j) {
+                    const bool refresh = ANYREF && ((mask >> j) & 1u);   // uniform over the grid
+                    FVec<VE> d;
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) {
+                        d.v[e] = __fsub_rn(vh[j].v[e], vs[j].v[e]);
+                        if (refresh) {
+                            float m = vm.v[e];
+                            delayed_nesterov<true>(vx.v[e], m, vc.v[e], d.v[e], eps, beta, inv_n, eps_n);
+                            vm.v[e] = m;
+                        } else {
+                            float m = 0.f;
+                            delayed_nesterov<false>(vx.v[e], m, vc.v[e], d.v[e], eps, beta, inv_n, eps_n);
+                        }
+                    }
+                    T::template store<VE, STREAM>(s0[j] + o, vx);
+                    if (STATS) {
+                        q_d[j] = sumsq<VE>(d);
+                        q_x[j] = sumsq<VE>(vx);
                     }
                 }
-                T::template store<VE, STREAM>(s0[j] + o, vx);
-            }
-            stf<VE, STREAM>(th + o, vx);
-            stf<VE, STREAM>(ac + o, vc);
-            if (ANYREF) stf<VE, STREAM>(ml + o, vm);
-            if (PUSH) {
-                FVec<VE> D;
+                stf<VE, STREAM>(th + o, vx);
+                stf<VE, STREAM>(ac + o, vc);
+                if (ANYREF) stf<VE, STREAM>(ml + o, vm);
+                if (PUSH) {
+                    FVec<VE> D;
 #pragma unroll
-                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
-                stf<VE, STREAM>(ob + o, D);
+                    for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                    stf<VE, STREAM>(ob + o, D);
+                    if (STATS) q_D = sumsq<VE>(D);
+                }
             }
+            if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, vb >> 5, lane, q_d, q_x, q_D);
         }
         done = nvec * VE;
     }
-    for (uint32_t i = done + threadIdx.x; i < c.count; i += TPB) {
-        float x = th[i], acc = ac[i], m = ANYREF ? ml[i] : 0.f;
+    for (uint32_t ib = done + warp32; ib < c.count; ib += TPB) {
+        const uint32_t i = ib + lane;
+        float q_d[NB], q_x[NB], q_D = 0.f;
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
-            const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
-            if (ANYREF && ((mask >> j) & 1u)) delayed_nesterov<true>(x, m, acc, d, eps, beta, inv_n, eps_n);
-            else {
-                float unused = 0.f;
-                delayed_nesterov<false>(x, unused, acc, d, eps, beta, inv_n, eps_n);
+        for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+        if (i < c.count) {
+            float x = th[i], acc = ac[i], m = ANYREF ? ml[i] : 0.f;
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const float d = __fsub_rn(T::load1(h[j] + i), T::load1(s0[j] + i));
+                if (ANYREF && ((mask >> j) & 1u)) delayed_nesterov<true>(x, m, acc, d, eps, beta, inv_n, eps_n);
+                else {
+                    float unused = 0.f;
+                    delayed_nesterov<false>(x, unused, acc, d, eps, beta, inv_n, eps_n);
+                }
+                T::store1(s0[j] + i, x);
+                if (STATS) {
+                    q_d[j] = fmaf(d, d, 0.f);
+                    q_x[j] = fmaf(x, x, 0.f);
+                }
             }
-            T::store1(s0[j] + i, x);
+            th[i] = x;
+            ac[i] = acc;
+            if (ANYREF) ml[i] = m;
+            if (PUSH) {
+                const float D = __fsub_rn(x, an[i]);
+                ob[i] = D;
+                if (STATS) q_D = fmaf(D, D, 0.f);
+            }
         }
-        th[i] = x;
-        ac[i] = acc;
-        if (ANYREF) ml[i] = m;
-        if (PUSH) ob[i] = __fsub_rn(x, an[i]);
+        if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, nrv + ((ib - done) >> 5), lane, q_d, q_x, q_D);
     }
+    if constexpr (STATS)
+        multi_stats_finish<NB, PUSH>(srow, nrv + ((c.count - done + 31u) >> 5), a.partial_delta, a.partial_theta, a.partial_Delta);
 }
 
 // =====================================================================================================
@@ -722,9 +910,12 @@ struct ArriveDeltaArgs {
     const float* anchor;
     float* outbox;
     float eta, beta, omb;
+    double* partial_delta;   // statistics, as in ArriveArgs
+    double* partial_Delta;
+    double* partial_theta;
 };
 
-template <class W, bool PUSH, bool STREAM, int VE>
+template <class W, bool PUSH, bool STATS, bool STREAM, int VE>
 __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 arrive_delta_kernel(const Chunk* __restrict__ chunks, ArriveDeltaArgs<W> a) {
     using T = WTraits<W>;
@@ -736,37 +927,88 @@ arrive_delta_kernel(const Chunk* __restrict__ chunks, ArriveDeltaArgs<W> a) {
     const float* an = PUSH ? a.anchor + c.begin : nullptr;
     float* ob = PUSH ? a.outbox + c.begin : nullptr;
     const float eta = a.eta, beta = a.beta, omb = a.omb;
+    __shared__ double srow[STATS ? 3 : 1][STATS ? kStatRows : 1];
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;
     uint32_t done = 0;
     if ((c.begin % VE) == 0) {
         const uint32_t nvec = c.count / VE;
-        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
-            const size_t o = (size_t)VE * v;
-            FVec<VE> vd = ldf<VE, STREAM>(dl + o);
-            FVec<VE> vx = ldf<VE, STREAM>(th + o);
-            FVec<VE> vm = ldf<VE, STREAM>(ml + o);
-            FVec<VE> va;
-            if (PUSH) va = ldf<VE, STREAM>(an + o);
+        nrv = (nvec + 31u) >> 5;
+        for (uint32_t vb = warp32; vb < nvec; vb += kThreads) {
+            const uint32_t v = vb + lane;
+            float q_d = 0.f, q_x = 0.f, q_D = 0.f;
+            if (v < nvec) {
+                const size_t o = (size_t)VE * v;
+                FVec<VE> vd = ldf<VE, STREAM>(dl + o);
+                FVec<VE> vx = ldf<VE, STREAM>(th + o);
+                FVec<VE> vm = ldf<VE, STREAM>(ml + o);
+                FVec<VE> va;
+                if (PUSH) va = ldf<VE, STREAM>(an + o);
 #pragma unroll
-            for (int e = 0; e < VE; ++e) model_update(vx.v[e], vm.v[e], vd.v[e], eta, beta, omb);
-            stf<VE, STREAM>(th + o, vx);
-            stf<VE, STREAM>(ml + o, vm);
-            T::template store<VE, STREAM>(s0 + o, vx);
-            if (PUSH) {
-                FVec<VE> D;
+                for (int e = 0; e < VE; ++e) model_update(vx.v[e], vm.v[e], vd.v[e], eta, beta, omb);
+                stf<VE, STREAM>(th + o, vx);
+                stf<VE, STREAM>(ml + o, vm);
+                T::template store<VE, STREAM>(s0 + o, vx);
+                if (STATS) {
+                    q_d = sumsq<VE>(vd);
+                    q_x = sumsq<VE>(vx);
+                }
+                if (PUSH) {
+                    FVec<VE> D;
 #pragma unroll
-                for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
-                stf<VE, STREAM>(ob + o, D);
+                    for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx.v[e], va.v[e]);
+                    stf<VE, STREAM>(ob + o, D);
+                    if (STATS) q_D = sumsq<VE>(D);
+                }
+            }
+            if (STATS) {
+                const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+                if (lane == 0) {
+                    srow[0][vb >> 5] = r_d;
+                    srow[1][vb >> 5] = r_x;
+                    if (PUSH) srow[2][vb >> 5] = r_D;
+                }
             }
         }
         done = nvec * VE;
     }
-    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
-        float x = th[j], m = ml[j];
-        model_update(x, m, dl[j], eta, beta, omb);
-        th[j] = x;
-        ml[j] = m;
-        T::store1(s0 + j, x);
-        if (PUSH) ob[j] = __fsub_rn(x, an[j]);
+    for (uint32_t jb = done + warp32; jb < c.count; jb += kThreads) {
+        const uint32_t j = jb + lane;
+        float q_d = 0.f, q_x = 0.f, q_D = 0.f;
+        if (j < c.count) {
+            const float d = dl[j];
+            float x = th[j], m = ml[j];
+            model_update(x, m, d, eta, beta, omb);
+            th[j] = x;
+            ml[j] = m;
+            T::store1(s0 + j, x);
+            if (STATS) {
+                q_d = fmaf(d, d, 0.f);
+                q_x = fmaf(x, x, 0.f);
+            }
+            if (PUSH) {
+                const float D = __fsub_rn(x, an[j]);
+                ob[j] = D;
+                if (STATS) q_D = fmaf(D, D, 0.f);
+            }
+        }
+        if (STATS) {
+            const uint32_t row = nrv + ((jb - done) >> 5);
+            const double r_d = row_sum(q_d), r_x = row_sum(q_x), r_D = PUSH ? row_sum(q_D) : 0.0;
+            if (lane == 0) {
+                srow[0][row] = r_d;
+                srow[1][row] = r_x;
+                if (PUSH) srow[2][row] = r_D;
+            }
+        }
+    }
+    if (STATS) {
+        __syncthreads();
+        const uint32_t nrows = nrv + ((c.count - done + 31u) >> 5);
+        if (threadIdx.x < (PUSH ? 3u : 2u)) {
+            double* dst = threadIdx.x == 0 ? a.partial_delta : threadIdx.x == 1 ? a.partial_theta : a.partial_Delta;
+            dst[blockIdx.x] = rows_total(srow[threadIdx.x], nrows);
+        }
     }
 }
 
@@ -787,10 +1029,13 @@ push_kernel(const Chunk* __restrict__ chunks, PushArgs a) {
     const float* th = a.th + c.begin;
     const float* an = a.anchor + c.begin;
     float* ob = a.outbox + c.begin;
-    float acc = 0.f;
+    __shared__ double srow[STATS ? kStatRows : 1];
+    const uint32_t lane = threadIdx.x & 31u, warp32 = threadIdx.x & ~31u;
+    uint32_t nrv = 0;
     uint32_t done = 0;
     if ((c.begin % VE) == 0) {
         const uint32_t nvec = c.count / VE;
+        nrv = (nvec + 31u) >> 5;
         for (uint32_t base = 0; base < nvec; base += kThreads * UNROLL) {
             FVec<VE> vx[UNROLL], va[UNROLL];
 #pragma unroll
@@ -804,26 +1049,41 @@ push_kernel(const Chunk* __restrict__ chunks, PushArgs a) {
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const uint32_t v = base + u * kThreads + threadIdx.x;
+                float q_D = 0.f;
                 if (v < nvec) {
                     FVec<VE> D;
 #pragma unroll
                     for (int e = 0; e < VE; ++e) D.v[e] = __fsub_rn(vx[u].v[e], va[u].v[e]);
                     stf<VE, STREAM>(ob + (size_t)VE * v, D);
-                    if (STATS) acc = sumsq<VE>(D, acc);
+                    if (STATS) q_D = sumsq<VE>(D);
+                }
+                if (STATS) {
+                    const uint32_t vb = base + u * kThreads + warp32;
+                    if (vb < nvec) {
+                        const double r = row_sum(q_D);
+                        if (lane == 0) srow[vb >> 5] = r;
+                    }
                 }
             }
         }
         done = nvec * VE;
     }
-    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
-        float D = __fsub_rn(th[j], an[j]);
-        ob[j] = D;
-        if (STATS) acc = fmaf(D, D, acc);
+    for (uint32_t jb = done + warp32; jb < c.count; jb += kThreads) {
+        const uint32_t j = jb + lane;
+        float q_D = 0.f;
+        if (j < c.count) {
+            float D = __fsub_rn(th[j], an[j]);
+            ob[j] = D;
+            if (STATS) q_D = fmaf(D, D, 0.f);
+        }
+        if (STATS) {
+            const double r = row_sum(q_D);
+            if (lane == 0) srow[nrv + ((jb - done) >> 5)] = r;
+        }
     }
     if (STATS) {
-        __shared__ double red[kThreads / 32];
-        double t = block_sum((double)acc, red);
-        if (threadIdx.x == 0) a.partial_Delta[blockIdx.x] = t;
+        __syncthreads();
+        if (threadIdx.x == 0) a.partial_Delta[blockIdx.x] = rows_total(srow, nrv + ((c.count - done + 31u) >> 5));
     }
 }
 
@@ -937,6 +1197,83 @@ pull_kernel(const Chunk* __restrict__ chunks, PullArgs a) {
 }
 
 // =====================================================================================================
+// GPS + PULL for the same LPS in one pass: the GPS receives Delta_l, and the answer Theta_i is merged
+// into that LPS at once (Alg. 1 lines 2-4 directly followed by lines 17-20 -- the order the event queue
+// produces when the two messages are adjacent, as on a fast link).  Theta_i is still in registers when
+// the merge needs it: 16 bytes read + 20 written per parameter instead of 24 + 16 for the two launches.
+// The in-flight snapshot (inbox) is still written, so the state equals that of the two launches bit for bit.
+// =====================================================================================================
+struct GpsPullArgs {
+    const float* outbox;
+    float* Theta;
+    float* Mg;
+    float* acc;      // delayed Nesterov only
+    float* inbox;
+    float* th;       // theta of the LPS
+    float* anchor;
+    float eta, beta, omb;          // paper rule
+    float inv_n, eps_n;            // delayed Nesterov (eta is its eps)
+    float alpha, oma;
+};
+
+// MODE 0: the paper's ModelUpdate; 1: delayed Nesterov, plain update; 2: delayed Nesterov, refresh update
+template <int MODE, bool STREAM, int VE>
+__global__ void __launch_bounds__(kThreads)
+gps_pull_kernel(const Chunk* __restrict__ chunks, GpsPullArgs a) {
+    const Chunk c = chunks[blockIdx.x];
+    const float* ob = a.outbox + c.begin;
+    float* Th = a.Theta + c.begin;
+    float* Mg = a.Mg + c.begin;
+    float* ac = MODE ? a.acc + c.begin : nullptr;
+    float* ib = a.inbox + c.begin;
+    float* th = a.th + c.begin;
+    float* an = a.anchor + c.begin;
+    const float eta = a.eta, beta = a.beta, omb = a.omb, inv_n = a.inv_n, eps_n = a.eps_n, alpha = a.alpha, oma = a.oma;
+    uint32_t done = 0;
+    if ((c.begin % VE) == 0) {
+        const uint32_t nvec = c.count / VE;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kThreads) {
+            const size_t o = (size_t)VE * v;
+            FVec<VE> vd = ldf<VE, STREAM>(ob + o);
+            FVec<VE> vx = ldf<VE, STREAM>(Th + o);
+            FVec<VE> vy = ldf<VE, STREAM>(th + o);
+            FVec<VE> vm, vc;
+            if (MODE != 1) vm = ldf<VE, STREAM>(Mg + o);
+            if (MODE) vc = ldf<VE, STREAM>(ac + o);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) {
+                if (MODE == 0) model_update(vx.v[e], vm.v[e], vd.v[e], eta, beta, omb);
+                else if (MODE == 1) {
+                    float unused = 0.f;
+                    delayed_nesterov<false>(vx.v[e], unused, vc.v[e], vd.v[e], eta, beta, inv_n, eps_n);
+                } else delayed_nesterov<true>(vx.v[e], vm.v[e], vc.v[e], vd.v[e], eta, beta, inv_n, eps_n);
+                vy.v[e] = merge(vy.v[e], vx.v[e], alpha, oma);
+            }
+            stf<VE, STREAM>(Th + o, vx);
+            if (MODE != 1) stf<VE, STREAM>(Mg + o, vm);
+            if (MODE) stf<VE, STREAM>(ac + o, vc);
+            stf<VE, STREAM>(ib + o, vx);
+            stf<VE, STREAM>(th + o, vy);
+            stf<VE, STREAM>(an + o, vy);
+        }
+        done = nvec * VE;
+    }
+    for (uint32_t j = done + threadIdx.x; j < c.count; j += kThreads) {
+        float x = Th[j], m = MODE != 1 ? Mg[j] : 0.f, acc = MODE ? ac[j] : 0.f;
+        if (MODE == 0) model_update(x, m, ob[j], eta, beta, omb);
+        else if (MODE == 1) delayed_nesterov<false>(x, m, acc, ob[j], eta, beta, inv_n, eps_n);
+        else delayed_nesterov<true>(x, m, acc, ob[j], eta, beta, inv_n, eps_n);
+        Th[j] = x;
+        if (MODE != 1) Mg[j] = m;
+        if (MODE) ac[j] = acc;
+        ib[j] = x;
+        const float r = merge(th[j], x, alpha, oma);
+        th[j] = r;
+        an[j] = r;
+    }
+}
+
+// =====================================================================================================
 // Initialisation helpers and statistics finalisation
 // =====================================================================================================
 // theta0[w] <- cast(Theta_0) for bf16 worker copies (Alg. 1 line 7)
@@ -946,9 +1283,47 @@ __global__ void cast_bf16_kernel(const float* __restrict__ src, uint16_t* __rest
     for (; i < n; i += stride) dst[i] = (uint16_t)bf16_narrow(src[i]);
 }
 
-// out[k] = sum of partial[c] over the chunks of tensor k, in a fixed order (one warp per tensor)
-__global__ void stats_finalize_kernel(const double* __restrict__ partial, const uint32_t* __restrict__ tensor_chunk_begin,
-                                      double* __restrict__ out, uint32_t n_tensors) {
+// Per-tensor statistics from per-chunk partial sums: one warp per (tensor, arrival of the launch, quantity)
+// adds the chunks of its tensor in a fixed order.  Quantity 0 = delta^2, 1 = theta^2, 2 = Delta^2.
+// The last arrival's sums go to `last` (what halos_stats reports for this LPS: [delta | Delta | theta][n_lps][nt]);
+// every arrival's sums go to record seq[j] of the caller's log (3 nt doubles: delta | theta | Delta, the
+// Delta part zero unless that arrival pushed) if the log has room for it.
+struct StatsFinalizeArgs {
+    const double* partial_delta;   // [nb][n_chunks]
+    const double* partial_theta;   // [nb][n_chunks]
+    const double* partial_Delta;   // [n_chunks]
+    const uint32_t* tensor_chunk_begin;
+    double* last;
+    double* log;
+    unsigned long long log_capacity;
+    unsigned long long seq[kMaxBatch];   // log record of each arrival of the launch
+    uint32_t n_chunks, n_tensors, n_lps, lps, nb;
+    int push;                      // the last arrival formed Delta
+};
+__global__ void stats_finalize_kernel(StatsFinalizeArgs a) {
+    const uint32_t k = blockIdx.x, j = blockIdx.y, q = blockIdx.z;
+    const bool is_last = j + 1 == a.nb;
+    const bool has_value = q < 2 || (is_last && a.push);
+    double v = 0.0;
+    if (has_value) {
+        const double* partial = q == 0 ? a.partial_delta + (size_t)j * a.n_chunks
+                              : q == 1 ? a.partial_theta + (size_t)j * a.n_chunks : a.partial_Delta;
+        const uint32_t b = a.tensor_chunk_begin[k], e = a.tensor_chunk_begin[k + 1];
+        for (uint32_t c = b + threadIdx.x; c < e; c += 32) v += partial[c];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    }
+    if (threadIdx.x != 0) return;
+    if (is_last && has_value) {
+        const uint32_t what = q == 0 ? 0u : q == 1 ? 2u : 1u;
+        a.last[((size_t)what * a.n_lps + a.lps) * a.n_tensors + k] = v;
+    }
+    if (a.log && a.seq[j] < a.log_capacity) a.log[((size_t)a.seq[j] * 3 + q) * a.n_tensors + k] = v;
+}
+
+// Delta^2 of a push launched on its own (halos_lps_push): out[k] = sum over the chunks of tensor k
+__global__ void stats_finalize_push_kernel(const double* __restrict__ partial, const uint32_t* __restrict__ tensor_chunk_begin,
+                                           double* __restrict__ out, uint32_t n_tensors) {
     const uint32_t k = blockIdx.x;
     if (k >= n_tensors) return;
     const uint32_t b = tensor_chunk_begin[k], e = tensor_chunk_begin[k + 1];

@@ -17,6 +17,7 @@ import oracle as oracle_mod
 from oracle import HalosOracle
 from paper_2506_04531_b200 import binding as hb
 from paper_2506_04531_b200.inputs import gen, trace as tr
+from paper_2506_04531_b200.inputs.gen_c import HostGenerator
 from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
 from paper_2506_04531_b200.inputs.layouts import Layout
 
@@ -40,17 +41,18 @@ def rel_error(got: np.ndarray, want: np.ndarray) -> float:
     return float(np.max(np.abs(g - o) / den))
 
 
-def default_probes(layout: Layout, width: int = 4096, n_random: int = 8, seed: int = 0) -> List[Tuple[int, int]]:
-    """First/last elements, a window around tensor boundaries, and random windows."""
+def default_probes(layout: Layout, width: int = 8192, n_random: int = 16, random_width: int = 65536, edge: int = 65536,
+                   seed: int = 0) -> List[Tuple[int, int]]:
+    """The first and last `edge` elements, `width` elements centred on EVERY tensor boundary, and `n_random`
+    random windows of `random_width` elements; overlapping windows are merged."""
     P = layout.P
     off = layout.offsets.astype(np.int64)
-    spans = [(0, min(P, 4 * width)), (max(0, P - 4 * width), P)]
-    step = max(1, (len(off) - 2) // 12)
-    for b in off[1:-1:step]:
-        spans.append((max(0, int(b) - width // 4), min(P, int(b) + width // 4)))
+    spans = [(0, min(P, edge)), (max(0, P - edge), P)]
+    for b in off[1:-1]:
+        spans.append((max(0, int(b) - width // 2), min(P, int(b) + width // 2)))
     rng = np.random.default_rng(seed)
-    for s in rng.integers(0, max(1, P - width), size=n_random):
-        spans.append((int(s), min(P, int(s) + width)))
+    for s in rng.integers(0, max(1, P - random_width), size=n_random):
+        spans.append((int(s), min(P, int(s) + random_width)))
     spans.sort()
     merged = []
     for lo, hi in spans:
@@ -73,11 +75,12 @@ class Lockstep:
         self.probes = probes if probes is not None else [(0, P)]
         self.full = probes is None
         self.dgen = DeviceGenerator(layout, seed, device=device, sigma_table=sigma_table)
+        self.hgen = HostGenerator(layout, seed, sigma_table=sigma_table)   # C twin of gen.py (cross-checked bit for bit)
         init_dev = self.dgen.theta_init()
         self.h = hb.Halos(init_dev, worker_lps, layout.numel, worker_dtype=worker_dtype, flags=flags,
                           chunk_elems=chunk_elems, **hyper)
         del init_dev
-        init_cpu = np.concatenate([gen.theta_init(layout, seed, lo, hi) for lo, hi in self.probes])
+        init_cpu = np.concatenate([self.hgen.theta_init(lo, hi) for lo, hi in self.probes])
         self.o = HalosOracle(init_cpu, worker_lps, worker_dtype=worker_dtype, dtype=np.float32, **hyper)
         if not self.full:
             idx = np.concatenate([np.arange(lo, hi, dtype=np.int64) for lo, hi in self.probes])
@@ -117,8 +120,7 @@ class Lockstep:
         s0 = self.o.buffer("th0", w)
         parts, pos = [], 0
         for lo, hi in self.probes:
-            parts.append(gen.worker_result(s0[pos:pos + hi - lo], self.layout, self.seed, w, rnd, lo, hi,
-                                           self.worker_dtype, sigma_table=self.sigma_table))
+            parts.append(self.hgen.worker_result(s0[pos:pos + hi - lo], w, rnd, lo, self.worker_dtype))
             pos += hi - lo
         return np.concatenate(parts)
 

@@ -543,3 +543,43 @@ def test_worker_staleness_bookkeeping():
         assert [o.worker_info(w)["round"] for w in range(len(wl))] == \
             [int(((events["kind"] == tr.ARRIVE) & (events["worker"] == w)).sum()) for w in range(len(wl))]
         o.close()
+
+
+# ----------------------------------------------------------------------------------------------
+# The event log (what the driver must report per event) derived from the oracle's counters, checked
+# against a direct count over the trace, and the stored hashes of the configured traces' logs
+# ----------------------------------------------------------------------------------------------
+def test_event_log_bookkeeping_and_golden_hashes():
+    from paper_2506_04531_b200.inputs import workloads
+    from sliced_oracle import log_hash, oracle_event_log
+    wl = workloads.workload("toy_k4")
+    ev = wl.trace()
+    log = oracle_event_log(wl, ev)
+    kind, lps = ev["kind"], ev["lps"]
+    t = [0] * wl.n_lps
+    t_last = [0] * wl.n_lps
+    answered_at = [0] * wl.n_lps
+    i = 0
+    for k in range(len(ev)):
+        l = int(lps[k])
+        if kind[k] == tr.ARRIVE:
+            t[l] += 1
+            assert int(log["pushed"][k]) == int(t[l] - t_last[l] == wl.K)       # Alg. 1 line 13
+        elif kind[k] == tr.GPS_RECV:
+            i += 1
+            answered_at[l] = i
+        else:
+            assert int(log["gps_lag"][k]) == i - answered_at[l]                 # GPS iterations since its Theta_i
+            t_last[l] = t[l]                                                     # line 18
+        assert (int(log["t"][k]), int(log["t_last"][k]), int(log["gps_iter"][k])) == (t[l], t_last[l], i)
+    assert int(log["pushed"].sum()) >= 20 and int(log["gps_lag"].max()) >= 1
+    golden = {}
+    for line in (Path(__file__).parent / "golden" / "event_log_hashes.txt").read_text().splitlines():
+        if line and not line.startswith("#"):
+            name, n, digest = line.split()
+            golden[name] = (int(n), digest)
+    assert set(golden) >= {"toy", "toy_k4", "70m", "160m", "410m"}
+    for name in ("toy", "toy_k4", "70m", "410m"):
+        w = workloads.workload(name)
+        e = w.trace()
+        assert (len(e), log_hash(oracle_event_log(w, e))) == golden[name], name
