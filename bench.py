@@ -170,9 +170,10 @@ class OracleReplayer:
         self.hg = HostGenerator(self.lay, wl.seed)
         init = self.hg.theta_init(0, self.S)
         self.o = HalosOracle(init, wl.worker_lps, worker_dtype=wl.worker_dtype, dtype=np.float32, **wl.hyper())
+        self.by_kind = {}
 
     def run(self, events, budget_s: float = float("inf")):
-        """Returns (seconds spent inside the oracle, events done)."""
+        """Returns (seconds spent inside the oracle, events done); self.by_kind accumulates [events, seconds] per kind."""
         from paper_2506_04531_b200.inputs import gen, trace as tr
         o, wl = self.o, self.wl
         spent, done = 0.0, 0
@@ -182,18 +183,29 @@ class OracleReplayer:
                 r = o.worker_info(w)["round"]
                 thH = self.hg.worker_result(o.buffer("th0", w), w, r, 0, wl.worker_dtype)   # untimed input
                 t0 = time.perf_counter()
-                o.arrive(w, thH)
+                pushed = o.arrive(w, thH)
+                name = "arrive_push" if pushed else "arrive"
             elif kind == tr.GPS_RECV:
                 t0 = time.perf_counter()
                 o.gps_recv(l)
+                name = "gps"
             else:
                 t0 = time.perf_counter()
                 o.pull(l)
-            spent += time.perf_counter() - t0
+                name = "pull"
+            dt = time.perf_counter() - t0
+            spent += dt
             done += 1
+            acc = self.by_kind.setdefault(name, [0, 0.0])
+            acc[0] += 1
+            acc[1] += dt
             if spent >= budget_s:
                 break
         return spent, done
+
+    def kind_rates(self):
+        """params/s per event kind from everything run so far."""
+        return {k: {"events": n, "value": n * self.S / t, "unit": UNIT} for k, (n, t) in sorted(self.by_kind.items()) if t > 0}
 
     def close(self):
         self.o.close()
@@ -214,14 +226,43 @@ def oracle_sample_all_cores(wl, events, slice_params: int, budget_s: float):
     return rate, cores
 
 
-def oracle_sample(wl, events, slice_params: int, budget_s: float):
+def oracle_sample(wl, events, slice_params: int, budget_s: float, want_kinds: bool = False):
     """Times the oracle from a fresh state on the first events of a trace until the time budget is used.
-    Returns (params/s, description, seconds, events)."""
+    Returns (params/s, description, seconds, events[, rates per event kind])."""
     rep = OracleReplayer(wl, slice_params)
     spent, done = rep.run(events, budget_s)
     S = rep.S
+    kinds = rep.kind_rates()
     rep.close()
-    return done * S / spent, f"first {done} events of the trace on the index slice [0,{S}) of {wl.layout.P} parameters", spent, done
+    out = (done * S / spent, f"first {done} events of the trace on the index slice [0,{S}) of {wl.layout.P} parameters", spent, done)
+    return out + (kinds,) if want_kinds else out
+
+
+def run_cpu_table(args):
+    """Oracle rates per event kind for every configuration: one core, and one replayer per core, each on bounded
+    index slices of the configured trace (CPU only; the core count is printed with the numbers)."""
+    from paper_2506_04531_b200.inputs import workloads
+    rows = {}
+    for name in ("toy", "70m", "160m", "410m"):
+        wl = workloads.workload(name)
+        ev = wl.trace()
+        budget = args.cpu_budget_s
+        rate, desc, spent, done, kinds = oracle_sample(wl, ev, 1 << 21, budget, want_kinds=True)
+        # long enough to contain pushes, GPS updates and merges: if the budget ended before the first round trip,
+        # time those kinds on the events around it
+        if "gps" not in kinds or "pull" not in kinds:
+            rep = OracleReplayer(wl, 1 << 18)
+            rep.run(ev[:min(len(ev), 400)])
+            small = rep.kind_rates()
+            rep.close()
+            for k in ("arrive_push", "gps", "pull"):
+                if k not in kinds and k in small:
+                    kinds[k] = dict(small[k], note="from a 256K-parameter slice")
+        all_rate, cores = oracle_sample_all_cores(wl, ev, 1 << 20, min(8.0, budget))
+        rows[name] = {"P": wl.layout.P, "one_core": {"value": rate, "unit": UNIT, "sample": desc + f" ({spent:.1f} s)"},
+                      "per_event_kind_one_core": kinds, "all_cores": {"value": all_rate, "cores": cores}}
+    print(json.dumps({"cpu_table": rows, "metric": METRIC, "kind": "oracle"}))
+    return 0
 
 
 # ------------------------------------------------------------------------------------ bandwidth sweep
@@ -298,6 +339,275 @@ def run_sweep(args):
     return 0
 
 
+# ------------------------------------------------------------------------------------ end-to-end leg
+def pcie_ceiling(torch, dev, nbytes: int, reps: int = 6):
+    """Pinned host<->device copies of one result's size, both directions at once on two streams (the shape of the
+    end-to-end leg): GB/s per direction.  Plain cudaMemcpyAsync through torch, no library code."""
+    hin = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    hout = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    din = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    dout = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    out = {}
+    for label, both in (("one_direction", False), ("both_directions", True)):
+        for timed in (False, True):
+            torch.cuda.synchronize(dev)
+            t0 = time.perf_counter()
+            for _ in range(reps if timed else 1):
+                with torch.cuda.stream(s1):
+                    din.copy_(hin, non_blocking=True)
+                if both:
+                    with torch.cuda.stream(s2):
+                        hout.copy_(dout, non_blocking=True)
+            torch.cuda.synchronize(dev)
+            dt = time.perf_counter() - t0
+        out["h2d_GBps_" + label] = reps * nbytes / 1e9 / dt
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        with torch.cuda.stream(s2):
+            hout.copy_(dout, non_blocking=True)
+    torch.cuda.synchronize(dev)
+    out["d2h_GBps_one_direction"] = reps * nbytes / 1e9 / (time.perf_counter() - t0)
+    return out
+
+
+def run_e2e(args, wl, hb, tr, torch, dist, dev, fresh_context, timed_events, arrive_slots, resident, eps, K, P, wbytes, wdt):
+    """The timed steps through the C ABI with HOST buffers: every arrival's result is copied in from pinned host
+    memory (halos_worker_delta_host) and every arrival's answer -- the model its worker restarts from -- is copied
+    out to pinned host memory (halos_worker_fetch_host); both copies are inside the timed region.  Covers as many
+    of the K steps as fit the pinned-memory budget."""
+    import psutil
+    budget = int(min(64 << 30, 0.35 * psutil.virtual_memory().available))
+    per_step = max(1, sum(1 for i in arrive_slots if i < eps))
+    steps = int(max(1, min(K, budget // (wbytes * P) // per_step)))
+    n_arr = sum(1 for i in arrive_slots if i < steps * eps)
+    host_results = torch.empty((n_arr, P), dtype=wdt).pin_memory()
+    host_results.copy_(resident[:n_arr])
+    ring = [torch.empty(P, dtype=wdt).pin_memory() for _ in range(4)]   # answers: a worker consumes its own at once
+    ceiling = pcie_ceiling(torch, dev, wbytes * P)
+    h = fresh_context()
+    torch.cuda.synchronize(dev)
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    n_out = 0
+    for s in range(steps):
+        win = timed_events[s * eps:(s + 1) * eps]
+        # results are copied in by the library; two staging buffers let the copy of the next result
+        # overlap the current update kernel, so up to two results are registered ahead
+        order = [k for k in range(len(win)) if int(win[k]["kind"]) == tr.ARRIVE]
+        ahead, fed = [], 0
+
+        def feed():
+            nonlocal fed
+            while fed < len(order) and len(ahead) < 2:
+                k = order[fed]
+                w = int(win[k]["worker"])
+                if any(int(win[p]["worker"]) == w for p in ahead):
+                    break
+                h.worker_delta_host(w, host_results[arrive_slots[s * eps + k]])
+                ahead.append(k)
+                fed += 1
+        for k in range(len(win)):
+            feed()
+            kind, l, w = int(win[k]["kind"]), int(win[k]["lps"]), int(win[k]["worker"])
+            if kind == tr.ARRIVE:
+                assert ahead and ahead[0] == k
+                ahead.pop(0)
+                if h.lps_apply(l, w):
+                    h.lps_push(l)
+                h.worker_fetch_host(w, ring[n_out % len(ring)])      # the step's result for this worker
+                n_out += 1
+            elif kind == tr.GPS_RECV:
+                h.gps_merge(l)
+            else:
+                h.lps_pull(l)
+    h.fetch_sync()
+    torch.cuda.synchronize(dev)
+    dt_ms = (time.perf_counter() - t0) * 1e3
+    u = float(steps * eps) * P
+    dt_ms, u_all = reduce_over_ranks(dist, dt_ms, u, dev)
+    h2d = int(n_arr / steps * P * wbytes)
+    d2h = int(n_out / steps * P * wbytes)
+    e2e = {"value": u_all / (dt_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "steps": steps, "ms_per_step": dt_ms / steps,
+           "what": "worker results from pinned host memory in, each worker's new start model to pinned host memory out"}
+    e2e["h2d_GBps"] = h2d / (e2e["ms_per_step"] * 1e6)
+    e2e["d2h_GBps"] = d2h / (e2e["ms_per_step"] * 1e6)
+    e2e["pcie_ceiling"] = ceiling      # plain pinned copies of one result's size, measured beside it
+    e2e["frac_of_pcie_ceiling"] = e2e["h2d_GBps"] / ceiling["h2d_GBps_both_directions"]
+    h.close()
+    del host_results, ring
+    return e2e
+
+
+# ------------------------------------------------------------------------------------ other configurations
+def config_kernel_table(name, args, torch, dev, peak):
+    """Per-kernel CUDA-event figures for a whole configured trace (every event, generator in the loop between
+    launches, L2 flushed after each generated input), once with one launch per event and once through the fused
+    driver.  The library's per-launch events do not need resident inputs."""
+    from paper_2506_04531_b200 import binding as hb
+    from paper_2506_04531_b200.inputs import gen, workloads
+    from paper_2506_04531_b200.inputs.gen_cuda import DeviceGenerator
+    wl = workloads.workload(name)
+    lay, P = wl.layout, wl.layout.P
+    wbytes = 4 if wl.worker_dtype == gen.F32 else 2
+    wdt = torch.float32 if wl.worker_dtype == gen.F32 else torch.int16
+    need = (2 + 5 * wl.n_lps) * 4 * P + 2 * wl.n_workers * wbytes * P + (3 << 30)
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    if need > free_b:
+        raise RuntimeError(f"needs {need / 1e9:.0f} GB of device memory, {free_b / 1e9:.0f} GB free")
+    events = wl.trace()
+    dg = DeviceGenerator(lay, wl.seed, device=dev)
+    bufs = [torch.empty(P, dtype=wdt, device=dev) for _ in range(wl.n_workers)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {"workload": f"{wl.name}: P={P}, {wl.n_workers} workers / {wl.n_lps} LPS, {('f32', 'bf16')[wl.worker_dtype]} copies, "
+                       f"whole trace of {len(events)} events", "l2": "256 MB written after each generated input"}
+    for label, mb in (("per_event", 1), ("fused", args.max_batch)):
+        h = hb.Halos(dg.theta_init(), wl.worker_lps, lay.numel, worker_dtype=wl.worker_dtype, chunk_elems=args.chunk_elems, **wl.hyper())
+
+        def producer(index, worker, rnd):
+            r = dg.worker_result(h.peek(hb.BUF_THETA0, worker), worker, rnd, out=bufs[worker], worker_dtype=wl.worker_dtype)
+            flush.zero_()
+            return r
+        h.replay(events[:64], producer, want_log=False, max_batch=mb)        # warm-up
+        h.timing_enable(True)
+        h.replay(events[64:], producer, want_log=False, max_batch=mb)
+        rec = h.timing_launches()
+        h.close()
+        table = kernel_table(rec, P)
+        for k in table.values():
+            if k["GBps"]:
+                k["frac_of_measured"] = k["GBps"] / peak
+                k["frac_of_8TBps"] = k["GBps"] / 8000.0
+        kernel_s = float(rec["ms"].astype(np.float64).sum()) * 1e-3
+        out[label] = {"kernels": {k: v for k, v in table.items() if v["launches"]},
+                      "params_per_s_kernel_time": float(rec["events"].sum()) * P / kernel_s}
+        del h
+    del bufs, flush
+    return out
+
+
+def run_kernel_table(args):
+    """CUDA-event GB/s of EVERY kernel of the library, including those the trace-driven runs rarely or never use
+    (standalone push, delayed-Nesterov plain/refresh, materialised deltas, every batch size 2..8, GPS+merge), on a
+    small-memory case: the 70M layout, 8 workers on one LPS, both worker dtypes.  Every buffer is larger than L2."""
+    import torch
+    from paper_2506_04531_b200 import binding as hb, build as _build
+    from paper_2506_04531_b200.inputs import gen, layouts, trace as tr
+    _build.build()
+    dev = torch.device("cuda", 0)
+    peak, peak_kind = measured_peak_gbs()
+    lay = layouts.named_layout("70m")
+    P = lay.P
+    rows = []
+
+    def add(label, wname, rec):
+        for k, name in enumerate(hb.KERNEL_NAMES):
+            r = rec[rec["kind"] == k]
+            for bpp in sorted(set(r["bytes_per_param"].tolist())):
+                q = r[r["bytes_per_param"] == bpp]
+                for nev in sorted(set(q["events"].tolist())):
+                    z = q[q["events"] == nev]
+                    ms = float(z["ms"].astype(np.float64).mean())
+                    gbps = bpp * P / 1e9 / (ms * 1e-3)
+                    rows.append({"case": label, "worker_dtype": wname, "kernel": name, "events_per_launch": int(nev),
+                                 "bytes_per_param": int(bpp), "launches": int(len(z)), "mean_us": ms * 1e3, "GBps": gbps,
+                                 "frac_of_measured": gbps / peak, "frac_of_8TBps": gbps / 8000.0})
+
+    for wdt, wname in ((gen.F32, "f32"), (gen.BF16, "bf16")):
+        tdt = torch.float32 if wdt == gen.F32 else torch.int16
+        init = torch.randn(P, device=dev) * 0.02
+        res = []
+        for w in range(8):
+            t = init + 1e-3 * torch.randn(P, device=dev)
+            res.append(t if wdt == gen.F32 else t.to(torch.bfloat16).view(torch.int16))
+        for label, kw in (("paper rule", {}),
+                          ("delayed Nesterov d_l=3 d_g=2", dict(optimizer=hb.OPT_DELAYED_NESTEROV, delay_l=3, delay_g=2, eta_l=0.6, eta_g=0.3)),
+                          ("materialised delta", dict(flags=hb.FLAG_MATERIALISE_DELTA)),
+                          ("statistics on", dict(flags=hb.FLAG_STATS))):
+            if "materialised" in label and kw.get("optimizer"):
+                continue
+            h = hb.Halos(init, [0] * 8, lay.numel, worker_dtype=wdt, K=1 << 20, **kw)
+            ev1 = np.zeros(1, dtype=tr.EVENT_DTYPE)
+
+            def calls():
+                # call by call: arrive, standalone push, GPS, merge, and the fused GPS+merge
+                for w in range(4):
+                    h.worker_delta(w, res[w])
+                    h.lps_apply(0, w)
+                h.lps_push(0); h.gps_merge(0); h.lps_pull(0)
+                h.lps_push(0); h.gps_merge_pull(0)
+                if "materialised" in label:
+                    return
+                # fused arrivals: batches of every size 2..8 (distinct workers), without and with a push
+                for nb in range(2, 9):
+                    ev = np.zeros(nb, dtype=tr.EVENT_DTYPE)
+                    ev["worker"] = np.arange(nb)
+                    h.replay(ev, lambda i, w, r: res[w], want_log=False, max_batch=nb)
+            calls()
+            torch.cuda.synchronize(dev)
+            h.timing_enable(True)
+            for _ in range(6):
+                calls()
+            add(label, wname, h.timing_launches())
+            h.close()
+        # pushes fused into the launch that closes a window: K = 1 (single arrival) and K = 4 (batch of four)
+        for Kw in (1, 4):
+            h = hb.Halos(init, [0] * 8, lay.numel, worker_dtype=wdt, K=Kw)
+            ev = np.zeros(Kw, dtype=tr.EVENT_DTYPE)
+            ev["worker"] = np.arange(Kw)
+            for rep in range(7):
+                if rep == 1:
+                    h.timing_enable(True)
+                h.replay(ev, lambda i, w, r: res[w], want_log=False, max_batch=Kw)
+                h.gps_merge_pull(0)
+            add(f"K={Kw} (Delta formed by the launch that closes the window)", wname, h.timing_launches())
+            h.close()
+        del res, init
+        torch.cuda.empty_cache()
+    print(json.dumps({"kernel_table": rows, "P": P, "peak_GBps": peak, "peak_source": peak_kind}))
+    return 0
+
+
+# ------------------------------------------------------------------------------------ shared by both arms
+RESIDENT_BUDGET_BYTES = 137 << 30     # worker results of the timed steps kept in HBM (a B200 has 180 GB; the state needs <= 25 GB)
+
+
+def events_per_step(wl, steps: int, asked: int) -> int:
+    """Step length: 128 events unless asked otherwise, cut down so that the results of all timed steps fit the
+    resident budget (~96% of the events are arrivals).  A function of the arguments only, so that both arms
+    of the benchmark replay the same windows."""
+    wbytes = 4 if wl.worker_dtype == 0 else 2
+    fit = RESIDENT_BUDGET_BYTES // (wbytes * wl.layout.P)
+    eps = asked if asked > 0 else 128
+    return int(max(1, min(eps, (fit * 100 // 96) // max(1, steps))))
+
+
+def spread(xs):
+    xs = [float(x) for x in xs]
+    return {"median": float(np.median(xs)), "min": min(xs), "max": max(xs), "n": len(xs),
+            "rel_spread": (max(xs) - min(xs)) / float(np.median(xs)) if xs and np.median(xs) else None}
+
+
+def kernel_table(records, P: int, elapsed_ms=None):
+    """Per kernel kind, from the library's per-launch records: launches, events carried out, mean duration and
+    achieved GB/s on the algorithmic bytes the library accounts for each launch."""
+    from paper_2506_04531_b200 import binding as hb
+    out = {}
+    for k, name in enumerate(hb.KERNEL_NAMES):
+        r = records[records["kind"] == k]
+        n = int(len(r))
+        ms = float(r["ms"].astype(np.float64).sum())
+        byts = float((r["bytes_per_param"].astype(np.float64) * P).sum())
+        out[name] = {"launches": n, "events": int(r["events"].sum()), "mean_ms": (ms / n if n else None),
+                     "bytes_per_param": (byts / P / n if n else None), "GBps": (byts / 1e9 / (ms * 1e-3) if n else None)}
+        if elapsed_ms:
+            out[name]["share_of_step"] = ms / elapsed_ms
+    return out
+
+
 # ------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -308,17 +618,26 @@ def main():
     ap.add_argument("--workload", default="160m", choices=["toy", "70m", "160m", "160m_dn", "410m", "70m_f32_small"])
     ap.add_argument("--events-per-step", type=int, default=0,
                     help="events per step; 0 = 128, reduced so that the results of all timed steps fit in HBM")
+    ap.add_argument("--repeats", type=int, default=5, help="how often each timed region is run (state rebuilt untimed in between)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-kernel tables of the other configurations")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--chunk-elems", type=int, default=0)
     ap.add_argument("--max-batch", type=int, default=8,
                     help="multi-event fusion in the driver: up to this many arrivals per launch (1 = one kernel per event)")
+    ap.add_argument("--launch-log", default="", help="write one record per timed launch of the reported run (.jsonl or .csv)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over buffer sizes instead of the default line")
     ap.add_argument("--sweep-max", type=int, default=0, help="largest size to include (0 = all)")
+    ap.add_argument("--kernel-table", action="store_true", help="CUDA-event GB/s of every kernel of the library on a 70M-size layout")
+    ap.add_argument("--cpu-table", action="store_true", help="oracle rates per event kind for every configuration (CPU only)")
     args = ap.parse_args()
     if args.sweep:
         return run_sweep(args)
+    if args.kernel_table:
+        return run_kernel_table(args)
+    if args.cpu_table:
+        return run_cpu_table(args)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
@@ -331,9 +650,10 @@ def main():
     lay = wl.layout
     P = lay.P
     wname = {0: "f32", 1: "bf16"}[wl.worker_dtype]
+    eps = events_per_step(wl, args.steps, args.events_per_step)
     config = {"workload": f"{wl.name}: decoder layout P={P} ({lay.n_tensors} tensors), {wl.n_workers} workers over "
                           f"{wl.n_lps} LPS, 1 GPS, fp32 master + {wname} worker copies, K={wl.K}, paper hyperparameters",
-              "events_per_step": args.events_per_step or 128, "trace_seed": wl.seed, "max_batch": args.max_batch,
+              "events_per_step": eps, "trace_seed": wl.seed, "max_batch": args.max_batch,
               "l2": "every buffer (%.0f MB) is larger than L2; no flush needed" % (P * 4 / 1e6),
               "parallelism": "index-sharded replicas, no collective" if world > 1 else "single GPU"}
 
@@ -341,15 +661,14 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        eps_ref = args.events_per_step or 128
-        events = window_events(args.steps + args.warmup, eps_ref, wl)
+        events = window_events(args.steps + args.warmup, eps, wl)
         # every step replays its whole window (the state carries over), on an index slice small enough
         # for the run to end within a few minutes
         S = min(1 << 22, P)
         rep = OracleReplayer(wl, S)
         t_total, total_done = 0.0, 0
         for s in range(args.steps + args.warmup):
-            win = events[s * eps_ref:(s + 1) * eps_ref]
+            win = events[s * eps:(s + 1) * eps]
             spent, done = rep.run(win)
             if s >= args.warmup:
                 t_total += spent
@@ -361,7 +680,7 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic", "config": config,
                 "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                 "sample": f"every step's {eps_ref} events on the index slice [0,{S}) of {P} parameters"},
+                                 "sample": f"every step's {eps} events on the index slice [0,{S}) of {P} parameters"},
                 "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "gpu_launches": 0}
         print(json.dumps(line))
@@ -395,22 +714,17 @@ def main():
     # The number of results that fit in HBM bounds the length of a step.
     wbytes = 4 if wl.worker_dtype == gen.F32 else 2
     wdt = torch.float32 if wl.worker_dtype == gen.F32 else torch.int16
-    n_state_bufs = 2 + 5 * wl.n_lps
-    state_bytes = n_state_bufs * 4 * P + wl.n_workers * wbytes * P
-    free_b, total_b = torch.cuda.mem_get_info(dev)
-    room = int(0.88 * (free_b - state_bytes - 3 * wbytes * P - (2 << 30)))
-    fit_arrivals = max(1, room // (wbytes * P))
-    eps = args.events_per_step if args.events_per_step > 0 else 128
-    eps = int(max(1, min(eps, (fit_arrivals * 100 // 96) // max(1, args.steps))))   # ~96% of the events are arrivals
     K, W = args.steps, args.warmup
     events = window_events(W + K, eps, wl)
     from paper_2506_04531_b200.inputs import trace as tr
     timed_events = events[W * eps:(W + K) * eps]
     arrive_slots = {int(i): n for n, i in enumerate(np.nonzero(timed_events["kind"] == tr.ARRIVE)[0])}
     n_timed_arrivals = len(arrive_slots)
-    if n_timed_arrivals > fit_arrivals:
-        raise SystemExit(f"{n_timed_arrivals} resident results do not fit in device memory (room for {fit_arrivals})")
-    config["events_per_step"] = eps
+    n_state_bufs = 2 + 5 * wl.n_lps + (1 + wl.n_lps if wl.optimizer else 0)
+    state_bytes = n_state_bufs * 4 * P + wl.n_workers * wbytes * P
+    free_b, total_b = torch.cuda.mem_get_info(dev)
+    if (n_timed_arrivals + 3) * wbytes * P + state_bytes + (2 << 30) > free_b:
+        raise SystemExit(f"{n_timed_arrivals} resident results do not fit in the {free_b / 1e9:.0f} GB of free device memory")
     config["inputs"] = (f"theta_H = theta_0 + sigma z per arrival (faithful), {n_timed_arrivals} results of the timed steps "
                         f"pre-generated by an untimed pass and resident in HBM ({n_timed_arrivals * wbytes * P / 1e9:.1f} GB)")
 
@@ -462,7 +776,7 @@ def main():
         h = fresh_context()
         torch.cuda.synchronize(dev)
         h.timing_enable(True)
-        launches0, batch0 = h.info()["launches"], h.batch_info()
+        launches0 = h.info()["launches"]
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(dev)
@@ -482,109 +796,75 @@ def main():
             dist.barrier()
         elapsed_ms = e0.elapsed_time(e1)
         launches = h.info()["launches"] - launches0
-        timing, batch1 = h.timing_read(), h.batch_info()
+        records = h.timing_launches()
         h.timing_enable(False)
         if state_digest(h) != want_digest:
             raise SystemExit("the timed run did not end in the state of the generating pass")
         h.close()
         units = float(K * eps) * P
         t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
-        n_multi = batch1["multi_launches"] - batch0["multi_launches"]
-        n_batched = batch1["batched_arrivals"] - batch0["batched_arrivals"]
-
-        def kernel_bytes(kind, n):
-            """algorithmic bytes of all timed launches of one kernel kind"""
-            if kind == "arrive_multi":
-                return (16 * n_multi + 3 * wbytes * n_batched) * P
-            return BYTES_PER_PARAM.get(kind, BYTES_PER_PARAM.get(kind + "_" + wname, 0)) * P * n
-
-        per_kernel = {k: {"launches": n, "mean_ms": (ms / n if n else None), "share_of_step": ms / elapsed_ms,
-                          "GBps": (kernel_bytes(k, n) / 1e9 / (ms * 1e-3) if n else None)} for k, (n, ms) in timing.items()}
-        dominant = max(timing, key=lambda k: timing[k][1])
-        dn, dms = timing[dominant]
-        d_bytes = kernel_bytes(dominant, dn) / dn
-        achieved = d_bytes / 1e9 / (dms / dn * 1e-3)
+        per_kernel = kernel_table(records, P, elapsed_ms)
+        dominant = max(per_kernel, key=lambda k: (per_kernel[k]["share_of_step"] or 0))
+        d = per_kernel[dominant]
+        d_bytes = d["bytes_per_param"] * P
         tpp = DRAM_BYTES_PER_PARAM.get(dominant + "_" + wname, DRAM_BYTES_PER_PARAM.get(dominant))
-        if dominant == "arrive_multi" and n_multi:
-            tpp = 15.24 + 3.0 * wbytes * n_batched / n_multi   # measured: model and momentum cross HBM once per batch
-        roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": achieved, "peak": peak,
-                    "unit": "GB/s", "frac": achieved / peak, "traffic": (tpp * P if tpp else None),
+        if dominant == "arrive_multi" and d["launches"]:
+            tpp = 15.24 + 3.0 * wbytes * d["events"] / d["launches"]   # measured: model and momentum cross HBM once per batch
+        roofline = {"bound": "hbm", "kernel": f"{dominant}_kernel<{wname}>", "achieved": d["GBps"], "peak": peak,
+                    "unit": "GB/s", "frac": d["GBps"] / peak, "traffic": (tpp * P if tpp else None),
                     "peak_source": f"of {peak_kind}", "algorithmic_bytes_per_launch": d_bytes, "per_kernel": per_kernel}
-        if n_multi:
-            roofline["arrivals_per_multi_launch"] = n_batched / n_multi
+        if dominant == "arrive_multi":
+            roofline["arrivals_per_multi_launch"] = d["events"] / d["launches"]
         return {"value": units_all / (t_ms * 1e-3), "ms_per_step": t_ms / K, "launches": int(launches),
-                "roofline": roofline, "clocks": clk.summary()}
+                "roofline": roofline, "clocks": clk.summary(), "records": records}
 
-    per_event = timed_region(1)                          # one kernel per event
-    main_run = timed_region(args.max_batch) if args.max_batch > 1 else per_event   # multi-event fusion in the driver
-    value, roofline, launches = main_run["value"], main_run["roofline"], main_run["launches"]
-    t_ms = main_run["ms_per_step"] * K
+    def repeated(max_batch):
+        """The region `--repeats` times (state rebuilt, untimed, in between); reports the median run with the spread."""
+        runs = [timed_region(max_batch) for _ in range(max(1, args.repeats))]
+        runs.sort(key=lambda r: r["value"])
+        med = runs[len(runs) // 2]
+        med["spread"] = {"value": spread([r["value"] for r in runs]),
+                         "dominant_kernel_GBps": spread([r["roofline"]["achieved"] for r in runs])}
+        reasons = sorted({x for r in runs for x in r["clocks"]["reasons"]})
+        med["clocks"] = dict(med["clocks"], reasons=reasons)
+        return med
 
-    # ---- end to end: the same steps with the results in pinned HOST memory ----
+    per_event = repeated(1)                               # one kernel per event: the per-event figure of the metric
+    fused = repeated(args.max_batch) if args.max_batch > 1 else None   # multi-event fusion in the driver
+    if args.launch_log and rank == 0:
+        from paper_2506_04531_b200 import metrics
+        metrics.write_launch_records(args.launch_log, per_event["records"], P)
+
+    # ---- end to end: the same steps with the results in pinned HOST memory and every arrival's answer
+    # (the model the worker restarts from, Alg. 1 line 12) copied back to pinned host memory ----
     e2e = None
     if not args.no_e2e:
-        e2e_steps = max(1, min(K, 3))
-        n_e2e_arr = sum(1 for i in arrive_slots if i < e2e_steps * eps)
-        host_results = torch.empty((n_e2e_arr, P), dtype=wdt).pin_memory()
-        host_results.copy_(resident[:n_e2e_arr])
-        probe = [(hb.BUF_THETA_G, 0)] + [(hb.BUF_THETA_L, l) for l in range(wl.n_lps)]
-        h = fresh_context()
-        torch.cuda.synchronize(dev)
-        if world > 1:
-            dist.barrier()
-        t0 = time.perf_counter()
-        d2h = 0
-        for s in range(e2e_steps):
-            win = timed_events[s * eps:(s + 1) * eps]
-            # results are copied in by the library; two staging buffers let the copy of the next result
-            # overlap the current update kernel, so up to two results are registered ahead
-            order = [k for k in range(len(win)) if int(win[k]["kind"]) == tr.ARRIVE]
-            ahead, fed = [], 0
-
-            def feed():
-                nonlocal fed
-                while fed < len(order) and len(ahead) < 2:
-                    k = order[fed]
-                    w = int(win[k]["worker"])
-                    if any(int(win[p]["worker"]) == w for p in ahead):
-                        break
-                    h.worker_delta_host(w, host_results[arrive_slots[s * eps + k]])
-                    ahead.append(k)
-                    fed += 1
-            for k in range(len(win)):
-                feed()
-                kind, l, w = int(win[k]["kind"]), int(win[k]["lps"]), int(win[k]["worker"])
-                if kind == tr.ARRIVE:
-                    assert ahead and ahead[0] == k
-                    ahead.pop(0)
-                    if h.lps_apply(l, w):
-                        h.lps_push(l)
-                elif kind == tr.GPS_RECV:
-                    h.gps_merge(l)
-                else:
-                    h.lps_pull(l)
-            # device -> host read of the step's result: a probe of the global and local models
-            d2h = sum(h.read(which, idx, 0, 1024).nbytes for which, idx in probe)
-        torch.cuda.synchronize(dev)
-        dt_ms = (time.perf_counter() - t0) * 1e3
-        u = float(e2e_steps * eps) * P
-        dt_ms, u_all = reduce_over_ranks(dist if world > 1 else None, dt_ms, u, dev)
-        e2e = {"value": u_all / (dt_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(n_e2e_arr / e2e_steps * P * wbytes), "d2h_bytes_per_step": int(d2h),
-               "steps": e2e_steps, "ms_per_step": dt_ms / e2e_steps}
-        e2e["h2d_GBps"] = e2e["h2d_bytes_per_step"] / (e2e["ms_per_step"] * 1e6)   # the PCIe copy bounds this leg
-        h.close()
-        del host_results
+        e2e = run_e2e(args, wl, hb, tr, torch, dist if world > 1 else None, dev, fresh_context, timed_events, arrive_slots,
+                      resident, eps, K, P, wbytes, wdt)
 
     del resident, scratch
     torch.cuda.empty_cache()
+
+    # ---- the other configurations: per-kernel figures over their whole traces (rank 0, N = 1 only) ----
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs:
+        configs = {}
+        for name in ("410m", "70m"):
+            if name == wl.name:
+                continue
+            try:
+                configs[name] = config_kernel_table(name, args, torch, dev, peak)
+            except Exception as e:              # e.g. not enough free memory for the 410M configuration
+                configs[name] = {"error": str(e)[:300]}
+            torch.cuda.empty_cache()
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_events = wl.trace()                     # the whole configured trace: the sample stops at the time budget
-        rate, desc, spent, done = oracle_sample(wl, cpu_events, 1 << 22, args.cpu_budget_s)
-        cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc + f" ({spent:.1f} s)"}
+        rate, desc, spent, done, per_kind = oracle_sample(wl, cpu_events, 1 << 22, args.cpu_budget_s, want_kinds=True)
+        cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc + f" ({spent:.1f} s)",
+               "per_event_kind": per_kind}
         try:
             all_rate, n_cores = oracle_sample_all_cores(wl, cpu_events, 1 << 20, min(6.0, args.cpu_budget_s))
             cpu["all_cores"] = {"value": all_rate, "cores": n_cores,
@@ -593,14 +873,21 @@ def main():
             cpu["all_cores"] = {"error": str(e)[:200]}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": t_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        def public(r):
+            return {k: v for k, v in r.items() if k != "records"}
+        line = {"metric": METRIC, "value": per_event["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": per_event["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-                "clocks": main_run["clocks"], "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "cpu_baseline": cpu,
-                "per_event_kernels": {"value": per_event["value"], "unit": UNIT, "ms_per_step": per_event["ms_per_step"],
-                                      "gpu_launches": per_event["launches"], "roofline": per_event["roofline"],
-                                      "note": "same workload with one kernel launch per event (max_batch = 1)"}}
+                "clocks": per_event["clocks"], "e2e": e2e, "gpu_launches": per_event["launches"],
+                "roofline": per_event["roofline"], "spread": per_event["spread"], "cpu_baseline": cpu,
+                "note": "value = one kernel launch per event (the per-event figure of the metric); fused_replay = the same "
+                        "events through the driver's multi-event fusion (bit-identical state, fewer bytes per event)"}
+        if fused is not None:
+            line["fused_replay"] = {"value": fused["value"], "unit": UNIT, "ms_per_step": fused["ms_per_step"],
+                                    "gpu_launches": fused["launches"], "roofline": fused["roofline"], "spread": fused["spread"],
+                                    "clocks": fused["clocks"]}
+        if configs is not None:
+            line["configs"] = configs
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

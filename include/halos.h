@@ -147,6 +147,16 @@ int halos_worker_delta(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_
  * cannot be allocated. */
 int halos_worker_delta_host(halos_ctx* ctx, uint32_t worker, const void* thetaH_flat_host);
 
+/* Alg. 1 line 12 seen from the worker: the model the worker restarts from, theta_{t,0} = cast(theta_t), as
+ * written by its last halos_lps_apply, copied to HOST memory (P elements of worker_dtype, packed).  The copy
+ * runs on a device-to-host stream the context owns, after the update that wrote the snapshot and before
+ * the next one that rewrites it (events order both), so it overlaps the update kernels and the host-to-device
+ * copies of halos_worker_delta_host.  dst_host is borrowed until halos_fetch_sync returns (pinned memory
+ * makes the copy asynchronous).  Launches a queued arrival of this worker first. */
+int halos_worker_fetch_host(halos_ctx* ctx, uint32_t worker, void* dst_host);
+/* Waits until every copy enqueued by halos_worker_fetch_host has landed in host memory. */
+int halos_fetch_sync(halos_ctx* ctx);
+
 /* Alg. 1 lines 10-13 at LPS `lps` for the pending result of `worker`:  t <- t+1;
  * theta_t <- ModelUpdate(theta_{t-1}, delta, eta_l, beta_l); the worker is scheduled theta_t
  * (theta0[worker] <- cast(theta_t)).  One fused kernel.  *push_due (may be NULL) receives
@@ -316,6 +326,20 @@ enum {
 };
 int halos_timing_enable(halos_ctx* ctx, int on);
 int halos_timing_read(halos_ctx* ctx, uint32_t kind, uint64_t* launches, double* total_ms);
+
+/* One record per launch timed since halos_timing_enable(ctx, 1), in launch order: its kind, how many trace
+ * events it carried out (a fused launch: several), its algorithmic traffic in bytes per parameter (every
+ * live buffer read once and written once: 16 + 3 w_b per arrival alone, 16 + 3 w_b n for n fused arrivals,
+ * +8 with Delta formed in the same pass, +8 for a momentum refresh under delayed Nesterov, 12 push, 24 GPS,
+ * 16 merge, 36 GPS+merge) and its duration.  Waits for the stream.  *n receives the number of launches
+ * timed; at most `capacity` records are written. */
+typedef struct halos_launch_record {
+    uint32_t kind;             /* HALOS_K_* */
+    uint32_t events;
+    uint32_t bytes_per_param;
+    float ms;
+} halos_launch_record;
+int halos_timing_launches(halos_ctx* ctx, halos_launch_record* out_host, uint64_t capacity, uint64_t* n);
 
 /* Push step for callers that must not allocate.  (The paper has no counterpart: this is a
  * deployment variant of Alg. 1 line 14 as computed by halos_lps_push with HALOS_FLAG_STATS.)

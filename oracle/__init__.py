@@ -31,17 +31,40 @@ OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1
 _WHICH = {"Theta": 0, "Mg": 1, "th": 2, "ml": 3, "anchor": 4, "outbox": 5, "inbox": 6, "th0": 7, "delta": 8, "acc": 9, "acc_g": 10}
 
 
+def _cpu_has(flag: str) -> bool:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("flags"):
+                return flag in line.split()
+    except OSError:
+        pass
+    return False
+
+
+def _isa_flags():
+    """-mfma where the host has the instruction: std::fma then compiles to one vfmadd instead of a libm call
+    (the same correctly rounded result, several times faster).  No other flag depends on the host."""
+    return ["-mfma"] if _cpu_has("fma") else []
+
+
+_FLAGS_NOTE = _HERE / "libhalos_oracle.flags"
+
+
 def build(force: bool = False) -> Path:
-    """Compile the oracle into a shared library next to its sources (idempotent)."""
+    """Compile the oracle into a shared library next to its sources (idempotent).  The library is rebuilt
+    when a source is newer or when it was built for instructions this host lacks."""
+    isa = _isa_flags()
     if not force and _LIB_PATH.exists():
         newest = max(p.stat().st_mtime for p in _SOURCES)
-        if _LIB_PATH.stat().st_mtime >= newest:
+        built_with = _FLAGS_NOTE.read_text().split() if _FLAGS_NOTE.exists() else None
+        if _LIB_PATH.stat().st_mtime >= newest and built_with is not None and set(built_with) <= set(isa):
             return _LIB_PATH
     tmp = _LIB_PATH.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+    cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", *isa, "-fPIC", "-shared",
            "-o", str(tmp), str(_SOURCES[0]), "-lpthread"]
     subprocess.run(cmd, check=True, cwd=str(_HERE))
     os.replace(tmp, _LIB_PATH)
+    _FLAGS_NOTE.write_text(" ".join(isa) + "\n")
     return _LIB_PATH
 
 

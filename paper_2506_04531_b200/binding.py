@@ -33,7 +33,8 @@ EXPORTED = (
     "halos_read", "halos_counters", "halos_worker_info", "halos_stats", "halos_info", "halos_timing_enable",
     "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
     "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards", "halos_replay_stream",
-    "halos_flush", "halos_gps_merge_pull", "halos_stats_log",
+    "halos_flush", "halos_gps_merge_pull", "halos_stats_log", "halos_worker_fetch_host", "halos_fetch_sync",
+    "halos_timing_launches",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -61,6 +62,8 @@ class Event(C.Structure):
     _fields_ = [("kind", C.c_uint8), ("lps", C.c_uint8), ("worker", C.c_uint16), ("pad", C.c_uint32),
                 ("time_ns", C.c_int64)]
 
+
+LAUNCH_RECORD_DTYPE = np.dtype([("kind", np.uint32), ("events", np.uint32), ("bytes_per_param", np.uint32), ("ms", np.float32)])
 
 EVENT_LOG_DTYPE = np.dtype([
     ("index", np.uint32), ("kind", np.uint8), ("lps", np.uint8), ("worker", np.uint16),
@@ -98,6 +101,9 @@ def load_library():
     lib.halos_lps_pull.argtypes = [vp, u32]
     lib.halos_gps_merge_pull.argtypes = [vp, u32]
     lib.halos_stats_log.argtypes = [vp, vp, u64]
+    lib.halos_worker_fetch_host.argtypes = [vp, u32, vp]
+    lib.halos_fetch_sync.argtypes = [vp]
+    lib.halos_timing_launches.argtypes = [vp, vp, u64, C.POINTER(u64)]
     lib.halos_destroy.argtypes = [vp]
     lib.halos_replay.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32)]
     lib.halos_replay_batched.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
@@ -274,6 +280,17 @@ class Halos:
         self._check(self._lib.halos_worker_delta_host(self._h, worker, _ptr(thetaH_host)))
         self._keep[worker] = thetaH_host
 
+    def worker_fetch_host(self, worker: int, dst_host):
+        """Copies the model the worker restarts from to a host tensor/array of the worker dtype (pinned memory makes
+        it asynchronous); complete after fetch_sync()."""
+        self._check(self._lib.halos_worker_fetch_host(self._h, worker, _ptr(dst_host)))
+        self._fetch_keep = getattr(self, "_fetch_keep", [])
+        self._fetch_keep.append(dst_host)
+
+    def fetch_sync(self):
+        self._check(self._lib.halos_fetch_sync(self._h))
+        self._fetch_keep = []
+
     def lps_apply(self, lps: int, worker: int) -> bool:
         due = C.c_int(0)
         self._check(self._lib.halos_lps_apply(self._h, lps, worker, C.byref(due)))
@@ -412,6 +429,15 @@ class Halos:
 
     def timing_enable(self, on: bool = True):
         self._check(self._lib.halos_timing_enable(self._h, int(on)))
+
+    def timing_launches(self) -> np.ndarray:
+        """Per-launch records (kind, events, bytes_per_param, ms) of everything timed since timing_enable(True)."""
+        n = C.c_uint64(0)
+        self._check(self._lib.halos_timing_launches(self._h, None, 0, C.byref(n)))
+        out = np.zeros(n.value, dtype=LAUNCH_RECORD_DTYPE)
+        if n.value:
+            self._check(self._lib.halos_timing_launches(self._h, out.ctypes.data, n.value, C.byref(n)))
+        return out
 
     def timing_read(self) -> dict:
         out = {}

@@ -44,6 +44,9 @@ struct WorkerState {
     uint64_t round = 0;    // arrivals applied so far
     uint64_t sched_t = 0;  // LPS counter when last scheduled
     cudaEvent_t table_copied = nullptr;  // guards reuse of the pinned pointer-table slot
+    cudaEvent_t snap_ready = nullptr;    // halos_worker_fetch_host: the snapshot to copy out has been written
+    cudaEvent_t fetched = nullptr;       // ... and the copy to the host has read it
+    bool fetch_outstanding = false;      // the next kernel that rewrites the snapshot must wait for `fetched`
     std::vector<uint8_t> vec_aligned;    // statistics contexts: per tensor, does the pending result allow the vector path
 };
 
@@ -65,6 +68,8 @@ struct Deferred {
 struct TimedLaunch {
     cudaEvent_t a, b;
     int kind;
+    uint32_t events;           // events of the trace this launch carried out
+    uint32_t bytes_per_param;  // its algorithmic traffic per parameter
 };
 
 }  // namespace
@@ -79,6 +84,7 @@ struct halos_ctx {
     std::vector<uint32_t> tensor_chunk_begin;
     cudaStream_t stream = nullptr;
     cudaStream_t copy_stream = nullptr;
+    cudaStream_t d2h_stream = nullptr;   // device-to-host copies of worker snapshots (created on first use)
 
     Chunk* d_chunks = nullptr;
     Chunk* d_chunks_rev = nullptr;  // the same table in reverse order
@@ -155,14 +161,21 @@ void release(halos_ctx* c) {
         cudaStreamSynchronize(c->copy_stream);
         cudaStreamDestroy(c->copy_stream);
     }
+    if (c->d2h_stream) {
+        cudaStreamSynchronize(c->d2h_stream);
+        cudaStreamDestroy(c->d2h_stream);
+    }
     for (void* p : c->owned) {
         if (c->cfg.free_ && c->cfg.alloc) c->cfg.free_(p, c->cfg.alloc_user);
         else cudaFree(p);
     }
     c->owned.clear();
     if (c->h_ptr_tables) cudaFreeHost((void*)c->h_ptr_tables);
-    for (auto& w : c->workers)
+    for (auto& w : c->workers) {
         if (w.table_copied) cudaEventDestroy(w.table_copied);
+        if (w.snap_ready) cudaEventDestroy(w.snap_ready);
+        if (w.fetched) cudaEventDestroy(w.fetched);
+    }
     for (int s = 0; s < kStageSlots; ++s) {
         if (c->stage_ready[s]) cudaEventDestroy(c->stage_ready[s]);
         if (c->stage_free[s]) cudaEventDestroy(c->stage_free[s]);
@@ -219,7 +232,10 @@ struct Timer {
     halos_ctx* c;
     cudaEvent_t a = nullptr, b = nullptr;
     int kind;
-    Timer(halos_ctx* c_, int kind_) : c(c_), kind(kind_) {
+    uint32_t events, bpp;
+    // events: trace events the launch carries out; bpp: bytes it must move per parameter (each live buffer read
+    // once and written once)
+    Timer(halos_ctx* c_, int kind_, uint32_t events_, uint32_t bpp_) : c(c_), kind(kind_), events(events_), bpp(bpp_) {
         nvtxRangePushA(kKindNames[kind]);
         if (!c->timing) return;
         if (!c->event_pool.empty()) {
@@ -237,7 +253,7 @@ struct Timer {
         nvtxRangePop();
         if (!a) return;
         cudaEventRecord(b, c->stream);
-        c->timed.push_back(TimedLaunch{a, b, kind});
+        c->timed.push_back(TimedLaunch{a, b, kind, events, bpp});
     }
 };
 
@@ -254,6 +270,14 @@ struct Timer {
     } while (0)
 
 inline bool stats_on(const halos_ctx* c) { return (c->cfg.flags & HALOS_FLAG_STATS) != 0; }
+
+// A kernel is about to rewrite this worker's snapshot: it must not overtake a copy of the old one to the host.
+int wait_fetch(halos_ctx* c, WorkerState& w) {
+    if (!w.fetch_outstanding) return HALOS_OK;
+    CU(c, cudaStreamWaitEvent(c->stream, w.fetched, 0));
+    w.fetch_outstanding = false;
+    return HALOS_OK;
+}
 
 template <class W>
 int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known) {
@@ -278,7 +302,7 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
     const bool refresh = refresh_known >= 0 ? refresh_known != 0 : ((s.t + 1) % c->cfg.delay_l) == 0;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     if (grid.x == 0) return HALOS_OK;
-    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE, 1, 16 + 3 * c->wb + (push ? 8 : 0) + (refresh ? 8 : 0));
     const Chunk* table = next_table(c);
     if (stats_on(c)) {
 #define CALL(R, P) arrive_dn_kernel<W, R, P, true, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a)
@@ -297,6 +321,10 @@ int launch_arrive_dn(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, b
 
 template <class W>
 int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool push, const void* flat, int refresh_known = -1) {
+    {
+        int rw = wait_fetch(c, w);
+        if (rw != HALOS_OK) return rw;
+    }
     if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) return launch_arrive_dn<W>(c, s, w, widx, push, flat, refresh_known);
     const bool stats = stats_on(c);
     if (w.pending == PEND_DELTA) {
@@ -304,7 +332,7 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
                              c->d_partial_delta, c->d_partial_Delta, c->d_partial_theta};
         const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
         if (grid.x == 0) return HALOS_OK;
-        Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+        Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE, 1, 20 + c->wb + (push ? 8 : 0));   // reads delta, not theta_H and theta_0
         const Chunk* table = next_table(c);
 #define CALL(P, S) arrive_delta_kernel<W, P, S, kStream, kVE><<<grid, block, 0, c->stream>>>(table, d)
         HALOS_PICK2(push, stats, CALL);
@@ -331,7 +359,7 @@ int launch_arrive(halos_ctx* c, LpsState& s, WorkerState& w, uint32_t widx, bool
     a.omb = 1.0f - c->cfg.beta_l;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     if (grid.x == 0) return HALOS_OK;
-    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE);
+    Timer tm(c, push ? HALOS_K_ARRIVE_PUSH : HALOS_K_ARRIVE, 1, 16 + 3 * c->wb + (push ? 8 : 0));
     const Chunk* table = next_table(c);
 #define CALL(P, S) arrive_kernel<W, P, S, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a)
     HALOS_PICK2(push, stats, CALL);
@@ -480,7 +508,7 @@ int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool pu
     constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     const bool any = a.refresh_mask != 0;
-    Timer tm(c, HALOS_K_ARRIVE_MULTI);
+    Timer tm(c, HALOS_K_ARRIVE_MULTI, NB, 16 + 3 * c->wb * NB + (push ? 8 : 0) + (any ? 8 : 0));
     const Chunk* table = next_table(c);
     if (stats_on(c)) {
 #define CALL(A, P) arrive_multi_dn_kernel<W, NB, A, P, true, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(table, a)
@@ -523,7 +551,7 @@ int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push)
     a.omb = 1.0f - c->cfg.beta_l;
     constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
-    Timer tm(c, HALOS_K_ARRIVE_MULTI);
+    Timer tm(c, HALOS_K_ARRIVE_MULTI, NB, 16 + 3 * c->wb * NB + (push ? 8 : 0));
     const Chunk* table = next_table(c);
 #define CALL(P, S) arrive_multi_kernel<W, NB, P, S, kStream, kVE, TPB><<<grid, block, 0, c->stream>>>(table, a)
     HALOS_PICK2(push, stats_on(c), CALL);
@@ -542,6 +570,8 @@ int flush_deferred_t(halos_ctx* c, uint32_t lps, std::vector<Deferred>& q, bool 
     if (q.empty()) return HALOS_OK;
     int rc = HALOS_OK;
     CU(c, cudaSetDevice(c->cfg.device));
+    for (const Deferred& d : q)
+        if ((rc = wait_fetch(c, c->workers[d.worker])) != HALOS_OK) return rc;
     switch (q.size()) {
         case 1: rc = launch_arrive<W>(c, s, c->workers[q[0].worker], q[0].worker, push, q[0].flat, q[0].refresh ? 1 : 0); break;
         case 2: rc = launch_arrive_multi<W, 2>(c, s, q.data(), push); break;
@@ -890,6 +920,34 @@ int halos_worker_delta_host(halos_ctx* c, uint32_t worker, const void* host) {
     return HALOS_OK;
 }
 
+int halos_worker_fetch_host(halos_ctx* c, uint32_t worker, void* dst_host) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (worker >= c->cfg.n_workers || !dst_host) return fail(c, HALOS_ERR_INVALID_ARG, "bad worker or null pointer");
+    {
+        int rq = flush_worker(c, worker);   // the snapshot is written by this worker's arrival, which may still be queued
+        if (rq != HALOS_OK) return rq;
+    }
+    WorkerState& w = c->workers[worker];
+    CU(c, cudaSetDevice(c->cfg.device));
+    if (!c->d2h_stream) CU(c, cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
+    if (!w.snap_ready) CU(c, cudaEventCreateWithFlags(&w.snap_ready, cudaEventDisableTiming));
+    if (!w.fetched) CU(c, cudaEventCreateWithFlags(&w.fetched, cudaEventDisableTiming));
+    CU(c, cudaEventRecord(w.snap_ready, c->stream));
+    CU(c, cudaStreamWaitEvent(c->d2h_stream, w.snap_ready, 0));
+    CU(c, cudaMemcpyAsync(dst_host, w.th0, c->P * c->wb, cudaMemcpyDeviceToHost, c->d2h_stream));
+    CU(c, cudaEventRecord(w.fetched, c->d2h_stream));
+    w.fetch_outstanding = true;
+    return HALOS_OK;
+}
+
+int halos_fetch_sync(halos_ctx* c) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (!c->d2h_stream) return HALOS_OK;
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->d2h_stream));
+    return HALOS_OK;
+}
+
 int halos_lps_apply(halos_ctx* c, uint32_t lps, uint32_t worker, int* push_due) {
     if (!c) return HALOS_ERR_INVALID_ARG;
     int rq = flush_all(c);
@@ -910,7 +968,7 @@ int halos_lps_push(halos_ctx* c, uint32_t lps) {
     PushArgs a{s.th, s.anchor, s.outbox, c->d_partial_Delta};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
     const bool stats = (c->cfg.flags & HALOS_FLAG_STATS) != 0;
-    Timer tm(c, HALOS_K_PUSH);
+    Timer tm(c, HALOS_K_PUSH, 0, 12);
     if (stats) push_kernel<true, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     else push_kernel<false, kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     tm.stop();
@@ -935,7 +993,8 @@ int halos_gps_merge(halos_ctx* c, uint32_t lps) {
     if (s.phase != HALOS_PUSHED) return fail(c, HALOS_ERR_BAD_STATE, "LPS %u has no Delta in flight", lps);
     CU(c, cudaSetDevice(c->cfg.device));
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
-    Timer tm(c, HALOS_K_GPS);
+    const bool gps_refresh = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV && ((c->gps_iter + 1) % c->cfg.delay_g) == 0;
+    Timer tm(c, HALOS_K_GPS, 1, 24 + (gps_refresh ? 8 : 0));
     if (c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV) {
         const float inv_n = 1.0f / (float)c->cfg.delay_g;
         GpsDnArgs a{s.outbox, c->Theta, c->Mg, c->acc_g, s.inbox, c->cfg.eta_g, c->cfg.beta_g, inv_n, c->cfg.eta_g * inv_n};
@@ -971,7 +1030,7 @@ static int pull_impl(halos_ctx* c, uint32_t lps) {
     CU(c, cudaSetDevice(c->cfg.device));
     PullArgs a{s.th, s.inbox, s.anchor, c->cfg.alpha, 1.0f - c->cfg.alpha};
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
-    Timer tm(c, HALOS_K_PULL);
+    Timer tm(c, HALOS_K_PULL, 1, 16);
     pull_kernel<kUnroll, kStream, kVE><<<grid, block, 0, c->stream>>>(next_table(c), a);
     tm.stop();
     c->launches++;
@@ -1004,7 +1063,8 @@ static int gps_pull_impl(halos_ctx* c, uint32_t lps) {
     a.alpha = c->cfg.alpha;
     a.oma = 1.0f - c->cfg.alpha;
     const dim3 grid((unsigned)c->chunks.size()), block(kThreads);
-    Timer tm(c, HALOS_K_GPS_PULL);
+    const bool gps_refresh = c->cfg.optimizer == HALOS_OPT_DELAYED_NESTEROV && ((c->gps_iter + 1) % c->cfg.delay_g) == 0;
+    Timer tm(c, HALOS_K_GPS_PULL, 2, 36 + (gps_refresh ? 8 : 0));
     const Chunk* table = next_table(c);
     if (c->cfg.optimizer != HALOS_OPT_DELAYED_NESTEROV) gps_pull_kernel<0, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a);
     else if (((c->gps_iter + 1) % c->cfg.delay_g) == 0) gps_pull_kernel<2, kStream, kVE><<<grid, block, 0, c->stream>>>(table, a);
@@ -1208,6 +1268,7 @@ int checkpoint(halos_ctx* c, const char* path, bool to_file) {
         if (w.pending != PEND_NONE) return fail(c, HALOS_ERR_BAD_STATE, "a worker result is registered but not applied");
     CU(c, cudaSetDevice(c->cfg.device));
     CU(c, cudaStreamSynchronize(c->stream));
+    if (c->d2h_stream) CU(c, cudaStreamSynchronize(c->d2h_stream));
     FILE* f = fopen(path, to_file ? "wb" : "rb");
     if (!f) return fail(c, HALOS_ERR_INVALID_ARG, "cannot open %s", path);
     void* bounce = nullptr;
@@ -1467,6 +1528,27 @@ int halos_timing_read(halos_ctx* c, uint32_t kind, uint64_t* launches, double* t
     }
     if (launches) *launches = n;
     if (total_ms) *total_ms = ms;
+    return HALOS_OK;
+}
+
+int halos_timing_launches(halos_ctx* c, halos_launch_record* out, uint64_t capacity, uint64_t* n_out) {
+    if (!c || (!out && capacity)) return HALOS_ERR_INVALID_ARG;
+    {
+        int rq = flush_all(c);
+        if (rq != HALOS_OK) return rq;
+    }
+    CU(c, cudaSetDevice(c->cfg.device));
+    CU(c, cudaStreamSynchronize(c->stream));
+    uint64_t n = 0;
+    for (auto& t : c->timed) {
+        if (n < capacity) {
+            float x = 0.f;
+            CU(c, cudaEventElapsedTime(&x, t.a, t.b));
+            out[n] = halos_launch_record{(uint32_t)t.kind, t.events, t.bytes_per_param, x};
+        }
+        n += 1;
+    }
+    if (n_out) *n_out = n;
     return HALOS_OK;
 }
 

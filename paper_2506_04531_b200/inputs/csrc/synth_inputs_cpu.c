@@ -39,21 +39,42 @@ static inline uint16_t bf16_narrow(float f) { /* round to nearest even, finite i
 }
 
 /* dtype 0 = fp32, 1 = bf16 patterns.  in may be NULL (then base_tbl[k] is the base).  tensor_off has
- * n_tensors + 1 entries; out/in cover the global indices [lo, lo + n). */
+ * n_tensors + 1 entries; out/in cover the global indices [lo, lo + n).  The range is walked tensor by tensor so
+ * that the inner loops have constant per-tensor factors and no control flow (they vectorise). */
 void halos_synth_fill_cpu(void* out, const void* in, int dtype, const float* base_tbl, const float* sigma_tbl,
                           const uint64_t* tensor_off, uint32_t n_tensors, uint64_t key, uint64_t lo, uint64_t n) {
     uint32_t k = 0;
-    while (k + 1 < n_tensors && tensor_off[k + 1] <= lo) ++k;
-    for (uint64_t j = 0; j < n; ++j) {
-        const uint64_t g = lo + j;
-        while (k + 1 < n_tensors && tensor_off[k + 1] <= g) ++k; /* last tensor that starts at or before g */
-        const float z = unit_noise(key, g);
-        float base;
-        if (in) base = dtype == 0 ? ((const float*)in)[j] : bf16_widen(((const uint16_t*)in)[j]);
-        else base = base_tbl[k];
-        const float prod = sigma_tbl[k] * z;
-        const float v = base + prod;
-        if (dtype == 0) ((float*)out)[j] = v;
-        else ((uint16_t*)out)[j] = bf16_narrow(v);
+    while (k + 1 < n_tensors && tensor_off[k + 1] <= lo) ++k; /* last tensor that starts at or before lo */
+    uint64_t j = 0;
+    while (j < n) {
+        const uint64_t g0 = lo + j;
+        while (k + 1 < n_tensors && tensor_off[k + 1] <= g0) ++k;
+        uint64_t seg = n - j; /* elements of [lo + j, lo + n) that belong to tensor k */
+        if (k + 1 < n_tensors && tensor_off[k + 1] - g0 < seg) seg = tensor_off[k + 1] - g0;
+        const float sigma = sigma_tbl[k], base_k = base_tbl[k];
+        if (dtype == 0) {
+            float* o = (float*)out + j;
+            const float* src = in ? (const float*)in + j : 0;
+            if (src) {
+                for (uint64_t i = 0; i < seg; ++i) {
+                    const float prod = sigma * unit_noise(key, g0 + i);
+                    o[i] = src[i] + prod;
+                }
+            } else {
+                for (uint64_t i = 0; i < seg; ++i) {
+                    const float prod = sigma * unit_noise(key, g0 + i);
+                    o[i] = base_k + prod;
+                }
+            }
+        } else {
+            uint16_t* o = (uint16_t*)out + j;
+            const uint16_t* src = in ? (const uint16_t*)in + j : 0;
+            for (uint64_t i = 0; i < seg; ++i) {
+                const float prod = sigma * unit_noise(key, g0 + i);
+                const float base = src ? bf16_widen(src[i]) : base_k;
+                o[i] = bf16_narrow(base + prod);
+            }
+        }
+        j += seg;
     }
 }

@@ -6,7 +6,9 @@ worker speeds, profiled step times of Pythia-70M/160M/410M on one H100: 238.4, 6
 """
 from __future__ import annotations
 
+import json
 from dataclasses import dataclass
+from pathlib import Path
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -73,20 +75,86 @@ class Workload:
         return hp
 
 
+CONFIG_DIR = Path(__file__).resolve().parent / "configs"
+_INT_KEYS = {"n_workers", "n_lps", "n_arrivals", "seed", "K", "delay_l", "delay_g"}
+_FLOAT_KEYS = {"t_profiled_ms", "eta_l", "beta_l", "eta_g", "beta_g", "alpha", "slow_region_factor", "bandwidth_scale"}
+_REQUIRED = ("name", "layout", "n_workers", "n_lps", "worker_dtype", "t_profiled_ms", "n_arrivals", "seed")
+
+
+def parse_config(text: str) -> dict:
+    """`key = value` lines ('#' starts a comment) or a JSON object -> dict of raw values."""
+    text = text.strip()
+    if text.startswith("{"):
+        return dict(json.loads(text))
+    out = {}
+    for n, line in enumerate(text.splitlines(), 1):
+        line = line.split("#", 1)[0].strip()
+        if not line:
+            continue
+        if "=" not in line:
+            raise ValueError(f"line {n}: expected key = value")
+        k, v = (x.strip() for x in line.split("=", 1))
+        if k in out:
+            raise ValueError(f"line {n}: {k} given twice")
+        out[k] = v
+    return out
+
+
+def from_config(cfg: dict) -> Workload:
+    """Builds a workload from a parsed configuration.  Keys: name, layout (toy | 70m | 160m | 410m | 1p4b, or
+    'decoder' with layers/d/vocab, or 'flat' with P), n_workers, n_lps, worker_dtype (f32 | bf16), t_profiled_ms,
+    n_arrivals, seed; optional K, eta_l, beta_l, eta_g, beta_g, alpha (default: the paper's selected values),
+    slow_region_factor, bandwidth_scale, dyn_updates, optimizer (paper | delayed_nesterov), delay_l, delay_g."""
+    cfg = dict(cfg)
+    missing = [k for k in _REQUIRED if k not in cfg]
+    if missing:
+        raise ValueError(f"configuration lacks {missing}")
+    lay = str(cfg.pop("layout"))
+    if lay == "decoder":
+        from .layouts import decoder_layout
+        layout = decoder_layout(str(cfg["name"]), int(cfg.pop("layers")), int(cfg.pop("d")), int(cfg.pop("vocab")))
+    elif lay == "flat":
+        from .layouts import flat_layout
+        layout = flat_layout(str(cfg["name"]), int(cfg.pop("P")))
+    else:
+        layout = named_layout(lay)
+    wd = str(cfg.pop("worker_dtype")).lower()
+    if wd not in ("f32", "bf16"):
+        raise ValueError("worker_dtype must be f32 or bf16")
+    kw = {}
+    for k, v in cfg.items():
+        if k == "name":
+            continue
+        if k in _INT_KEYS:
+            kw[k] = int(v)
+        elif k in _FLOAT_KEYS:
+            kw[k] = float(v)
+        elif k == "dyn_updates":
+            kw[k] = str(v).lower() in ("1", "true", "yes")
+        elif k == "optimizer":
+            kw[k] = {"paper": 0, "delayed_nesterov": 1}[str(v)]
+        else:
+            raise ValueError(f"unknown configuration key {k!r}")
+    n_workers, n_lps = kw.pop("n_workers"), kw.pop("n_lps")
+    if n_workers % n_lps:
+        raise ValueError("n_workers must be a multiple of n_lps")
+    return Workload(str(cfg["name"]), layout, n_workers, n_lps, gen.F32 if wd == "f32" else gen.BF16,
+                    kw.pop("t_profiled_ms"), kw.pop("n_arrivals"), **kw)
+
+
+def load(path) -> Workload:
+    """A workload from a configuration file (key = value lines or JSON)."""
+    return from_config(parse_config(Path(path).read_text()))
+
+
 def workload(name: str) -> Workload:
     """toy | toy_k4 | 70m | 160m | 160m_dn | 410m | 70m_f32_small | paper_cluster | paper_cluster_small |
-    hetero_grouping_small  (hyperparameters: the paper's selected values)."""
-    if name == "toy":
-        return Workload("toy", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1)
+    hetero_grouping_small  (hyperparameters: the paper's selected values).  The four benchmark configurations
+    toy, 70m, 160m and 410m are read from the files in configs/."""
+    if name in ("toy", "70m", "160m", "410m"):
+        return load(CONFIG_DIR / f"{name}.cfg")
     if name == "toy_k4":
         return Workload("toy_k4", named_layout("toy"), 4, 2, gen.F32, 10.0, 200, seed=1, K=4)
-    if name == "70m":
-        return Workload("70m", named_layout("70m"), 8, 2, gen.BF16, 238.4, 1000, seed=2)
-    if name == "160m":
-        return Workload("160m", named_layout("160m"), 16, 4, gen.F32, 623.0, 2000, seed=3)
-    if name == "410m":
-        return Workload("410m", named_layout("410m"), 32, 4, gen.F32, 1589.7, 2000, seed=4,
-                        slow_region_factor=3.0)
     if name == "160m_dn":
         # the 160M configuration under the optimizer and the selected values of the paper's experiments:
         # delayed Nesterov with d_l = 16, eta_l = 16 x 0.2, d_g = 2, eta_g = 2 x 0.15

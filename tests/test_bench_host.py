@@ -114,3 +114,22 @@ def test_index_sharded_replicas_gloo(tmp_path):
     half = P // 2
     want = np.concatenate([o.buffer("Theta")[:half], o.buffer("th", 1)[:half], o.buffer("Theta")[half:], o.buffer("th", 1)[half:]])
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_step_length_is_shared_by_both_arms_and_kernel_table():
+    import bench
+    from paper_2506_04531_b200 import binding as hb
+    from paper_2506_04531_b200.inputs import workloads
+    wl = workloads.workload("160m")
+    # a function of the arguments only (never of the free memory of whichever machine runs the arm)
+    assert bench.events_per_step(wl, 20, 0) == bench.events_per_step(wl, 20, 0) == 11
+    assert bench.events_per_step(wl, 10, 0) == 23 and bench.events_per_step(wl, 10, 8) == 8
+    assert bench.events_per_step(workloads.workload("toy"), 10, 0) == 128
+    rec = np.zeros(4, dtype=hb.LAUNCH_RECORD_DTYPE)
+    rec["kind"], rec["events"], rec["bytes_per_param"], rec["ms"] = [0, 0, 5, 6], [1, 1, 3, 2], [28, 36, 52, 36], [1.0, 1.0, 2.0, 1.0]
+    t = bench.kernel_table(rec, 10 ** 9, elapsed_ms=10.0)
+    assert t["arrive"]["launches"] == 2 and t["arrive"]["bytes_per_param"] == 32.0 and abs(t["arrive"]["GBps"] - 32000.0) < 1e-6
+    assert t["arrive_multi"]["events"] == 3 and abs(t["arrive_multi"]["GBps"] - 26000.0) < 1e-6
+    assert t["gps_pull"]["share_of_step"] == 0.1 and t["push"]["launches"] == 0 and t["push"]["GBps"] is None
+    s = bench.spread([3.0, 1.0, 2.0])
+    assert (s["median"], s["min"], s["max"], s["n"]) == (2.0, 1.0, 3.0, 3) and s["rel_spread"] == 1.0

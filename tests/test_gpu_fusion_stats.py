@@ -175,14 +175,14 @@ def test_statistics_inside_fused_launches(mode):
         log = torch.full((n_arr + 3, 3, lay.n_tensors), -1.0, dtype=torch.float64, device="cuda")
         h.stats_log(log)
         if mode == "pointer_tables":
-            # per-tensor result buffers; every second worker's odd tensors are shifted by one element, so workers
+            # per-tensor result buffers; the odd tensors of workers 4..7 are shifted by one element, so workers
             # differ in which tensors may take the vector path (such arrivals must not share a launch)
             off = lay.offsets.astype(np.int64)
             parts = []
             for w in range(len(worker_lps)):
                 row = []
                 for k, n in enumerate(lay.numel):
-                    pad = 1 if (w % 2 == 1 and k % 2 == 1) else 0
+                    pad = 1 if (4 <= w < 8 and k % 2 == 1) else 0
                     row.append(torch.empty(int(n) + pad + 8, dtype=tdt, device="cuda")[pad:pad + int(n)])
                 parts.append(row)
 
@@ -293,3 +293,41 @@ def test_cuda_path_on_index_shards_equals_unsharded(wdt):
             assert np.array_equal(glued.view(np.uint8), full.read(which, idx).view(np.uint8)), (which, idx)
     for h in shards + [full]:
         h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the worker's new start model copied to host memory, overlapping later updates
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt", [gen.F32, gen.BF16])
+def test_worker_fetch_host_returns_the_scheduled_model(wdt):
+    lay = layouts.ragged_layout("r", [300_001, 33, 2_000_003, 5, 65536])
+    worker_lps = [0, 0, 1]
+    hp = dict(PAPER_HP, K=3)
+    events = tr.random_trace(worker_lps, 40, 3, seed=13)
+    dg = DeviceGenerator(lay, 59)
+    h = hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, **hp)
+    o = HalosOracle(gen.theta_init(lay, 59), worker_lps, worker_dtype=wdt, **hp)
+    prod = _producer(h, dg, lay, worker_lps, wdt)
+    np_dt = np.float32 if wdt == gen.F32 else np.uint16
+    t_dt = torch.float32 if wdt == gen.F32 else torch.int16
+    outs, wants = [], []
+    for n, ev in enumerate(events):
+        kind, l, w = int(ev["kind"]), int(ev["lps"]), int(ev["worker"])
+        h.replay(events[n:n + 1], prod, max_batch=8, keep_queued=True)    # arrivals may stay queued: fetch launches them
+        if kind == tr.ARRIVE:
+            o.arrive(w, gen.worker_result(o.buffer("th0", w), lay, 59, w, o.worker_info(w)["round"], worker_dtype=wdt))
+            dst = torch.empty(lay.P, dtype=t_dt).pin_memory()
+            h.worker_fetch_host(w, dst)          # not waited for: later updates (of this worker too) run on
+            outs.append(dst)
+            wants.append(o.buffer("th0", w).copy())
+        elif kind == tr.GPS_RECV:
+            o.gps_recv(l)
+        else:
+            o.pull(l)
+    h.flush()
+    h.fetch_sync()
+    assert len(outs) >= 25
+    for dst, want in zip(outs, wants):
+        assert np.array_equal(dst.numpy().view(np_dt), want.view(np_dt))
+    h.close()
+    o.close()

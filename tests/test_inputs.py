@@ -179,3 +179,50 @@ def test_trace_file_round_trip(tmp_path):
     (tmp_path / "junk").write_bytes(bytes(range(32)))
     with pytest.raises(ValueError):
         tr.load_trace(tmp_path / "junk")
+
+
+def test_configuration_files_and_reader(tmp_path):
+    """The four benchmark configurations are read from key = value files; the reader takes JSON too and
+    refuses unknown keys, missing keys and bad values."""
+    import json
+    import pytest
+    from paper_2506_04531_b200.inputs import workloads as W
+    want = {"toy": (1 << 20, 4, 2, gen.F32, 200, 1), "70m": (70_426_624, 8, 2, gen.BF16, 1000, 2),
+            "160m": (162_322_944, 16, 4, gen.F32, 2000, 3), "410m": (405_334_016, 32, 4, gen.F32, 2000, 4)}
+    for name, (P, nw, nl, wd, na, seed) in want.items():
+        wl = W.workload(name)
+        assert (wl.layout.P, wl.n_workers, wl.n_lps, wl.worker_dtype, wl.n_arrivals, wl.seed) == (P, nw, nl, wd, na, seed)
+        assert wl.hyper() == dict(eta_l=0.2, beta_l=0.9, eta_g=0.15, beta_g=0.5, alpha=0.25, K=32)
+    assert W.workload("410m").slow_region_factor == 3.0
+    cfg = dict(name="x", layout="decoder", layers=2, d=64, vocab=300, n_workers=6, n_lps=3, worker_dtype="bf16",
+               t_profiled_ms=5.0, n_arrivals=40, seed=9, K=4, alpha=0.5, optimizer="delayed_nesterov", delay_l=3, delay_g=2)
+    (tmp_path / "x.json").write_text(json.dumps(cfg))
+    (tmp_path / "x.cfg").write_text("\n".join(f"{k} = {v}  # note" for k, v in cfg.items()))
+    a, b = W.load(tmp_path / "x.json"), W.load(tmp_path / "x.cfg")
+    assert a == b and a.layout.n_tensors == 28 and a.worker_dtype == gen.BF16 and a.hyper()["delay_l"] == 3
+    assert a.worker_lps == [0, 0, 1, 1, 2, 2] and len(a.trace()) >= 40
+    for bad in (dict(cfg, colour="red"), {k: v for k, v in cfg.items() if k != "seed"}, dict(cfg, worker_dtype="f16"),
+                dict(cfg, n_workers=7)):
+        with pytest.raises((ValueError, KeyError)):
+            W.from_config(bad)
+    with pytest.raises(ValueError):
+        W.parse_config("K 4")
+
+
+def test_metrics_sinks(tmp_path):
+    import csv
+    import json
+    from paper_2506_04531_b200 import binding as hb, metrics
+    rec = np.zeros(3, dtype=hb.LAUNCH_RECORD_DTYPE)
+    rec["kind"], rec["events"], rec["bytes_per_param"], rec["ms"] = [0, 5, 6], [1, 4, 2], [28, 64, 36], [0.5, 1.0, 0.25]
+    assert metrics.write_launch_records(tmp_path / "l.jsonl", rec, 1000) == 3
+    rows = [json.loads(x) for x in (tmp_path / "l.jsonl").read_text().splitlines()]
+    assert rows[1] == {"launch": 1, "kernel": "arrive_multi", "events": 4, "bytes": 64000, "us": 1000.0, "GBps": 64000 / 1e9 / 1e-3}
+    metrics.write_launch_records(tmp_path / "l.csv", rec, 1000)
+    got = list(csv.DictReader(open(tmp_path / "l.csv")))
+    assert [r["kernel"] for r in got] == ["arrive", "arrive_multi", "gps_pull"]
+    log = np.zeros(2, dtype=hb.EVENT_LOG_DTYPE)
+    log["kind"], log["t"], log["fused"] = [0, 2], [7, 7], [1, 0]
+    metrics.write_event_log(tmp_path / "e.jsonl", log)
+    ev = [json.loads(x) for x in (tmp_path / "e.jsonl").read_text().splitlines()]
+    assert ev[0]["kind"] == "ARRIVE" and ev[1]["kind"] == "PULL" and ev[0]["t"] == 7 and ev[0]["fused"] == 1
