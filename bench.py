@@ -376,9 +376,9 @@ def run_e2e(args, wl, hb, tr, torch, dist, dev, fresh_context, timed_events, arr
     """The timed steps through the C ABI with HOST buffers: every arrival's result is copied in from pinned host
     memory (halos_worker_delta_host) and every arrival's answer -- the model its worker restarts from -- is copied
     out to pinned host memory (halos_worker_fetch_host); both copies are inside the timed region.  Covers as many
-    of the K steps as fit the pinned-memory budget."""
+    of the K steps as fit the pinned-memory budget (min(128 GB, 60% of the free host memory))."""
     import psutil
-    budget = int(min(64 << 30, 0.35 * psutil.virtual_memory().available))
+    budget = int(min(128 << 30, 0.6 * psutil.virtual_memory().available))
     per_step = max(1, sum(1 for i in arrive_slots if i < eps))
     steps = int(max(1, min(K, budget // (wbytes * P) // per_step)))
     n_arr = sum(1 for i in arrive_slots if i < steps * eps)

@@ -505,7 +505,7 @@ int launch_arrive_multi_dn(halos_ctx* c, LpsState& s, const Deferred* d, bool pu
     a.beta = c->cfg.beta_l;
     a.inv_n = 1.0f / (float)c->cfg.delay_l;
     a.eps_n = c->cfg.eta_l * a.inv_n;
-    constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
+    constexpr int TPB = multi_dn_threads<NB>();
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     const bool any = a.refresh_mask != 0;
     Timer tm(c, HALOS_K_ARRIVE_MULTI, NB, 16 + 3 * c->wb * NB + (push ? 8 : 0) + (any ? 8 : 0));
@@ -549,7 +549,7 @@ int launch_arrive_multi(halos_ctx* c, LpsState& s, const Deferred* d, bool push)
     a.eta = c->cfg.eta_l;
     a.beta = c->cfg.beta_l;
     a.omb = 1.0f - c->cfg.beta_l;
-    constexpr int TPB = NB <= 2 ? kThreads : kMultiWideThreads;
+    constexpr int TPB = multi_threads<NB>();
     const dim3 grid((unsigned)c->chunks.size()), block(TPB);
     Timer tm(c, HALOS_K_ARRIVE_MULTI, NB, 16 + 3 * c->wb * NB + (push ? 8 : 0));
     const Chunk* table = next_table(c);

@@ -391,6 +391,35 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
 constexpr int kMaxBatch = 8;
 constexpr int kMultiWideThreads = 256;   // CTA size of the multi-arrival kernel for batches of 3..8 (register budget)
 
+// Resident CTAs per SM the fused kernels are compiled for (it bounds the registers per thread).  Batches of
+// 5..8 fp32 results keep 2 NB + 2 vectors of 32 B in flight per thread and saturate HBM with ONE CTA of 256
+// threads per SM; bf16 results are half as wide, one CTA does not keep enough bytes in flight, so those
+// kernels are compiled for two (128 registers, a few spilled to L1).
+#ifndef HALOS_WIDE_MINBLOCKS_BF16
+#define HALOS_WIDE_MINBLOCKS_BF16 2
+#endif
+// CTA size / resident CTAs of the delayed-Nesterov kernel for batches of 2 (one more stream than the paper rule).
+#ifndef HALOS_DN2_THREADS
+#define HALOS_DN2_THREADS 256
+#endif
+#ifndef HALOS_DN2_MINBLOCKS
+#define HALOS_DN2_MINBLOCKS 3
+#endif
+#ifndef HALOS_WIDE_MINBLOCKS_BF16_STATS
+#define HALOS_WIDE_MINBLOCKS_BF16_STATS 2
+#endif
+template <class W, int NB, int TPB, bool STATS = false>
+constexpr int multi_min_blocks() {
+    return NB <= 2 ? 1024 / TPB
+                   : (NB <= 4 ? 512 / TPB : (sizeof(W) == 2 ? (STATS ? HALOS_WIDE_MINBLOCKS_BF16_STATS : HALOS_WIDE_MINBLOCKS_BF16) : 1));
+}
+template <int NB> constexpr int multi_threads() { return NB <= 2 ? kThreads : kMultiWideThreads; }
+template <int NB> constexpr int multi_dn_threads() { return NB <= 2 ? HALOS_DN2_THREADS : kMultiWideThreads; }
+template <class W, int NB, int TPB, bool STATS = false>
+constexpr int multi_dn_min_blocks() {
+    return NB <= 2 ? HALOS_DN2_MINBLOCKS : multi_min_blocks<W, NB, TPB, STATS>();
+}
+
 template <class W>
 struct ArriveMultiArgs {
     const W* h_flat[kMaxBatch];          // per arrival: flat result ...
@@ -408,21 +437,20 @@ struct ArriveMultiArgs {
 };
 
 // Statistics of a fused launch: quantity 2j = delta^2 of arrival j, 2j+1 = theta^2 after arrival j, 2 NB = Delta^2.
+// Every lane of the warp calls this (lanes without an item pass 0).
+__device__ __forceinline__ void stats_row_put(double* rows, uint32_t row, uint32_t lane, float item) {
+    const double r = row_sum(item);
+    if (lane == 0) rows[row] = r;
+}
 template <int NB, bool PUSH>
 __device__ __forceinline__ void multi_stats_rows(double (*srow)[kStatRows + 1], uint32_t row, uint32_t lane,
                                                  const float* q_d, const float* q_x, float q_D) {
 #pragma unroll
     for (int j = 0; j < NB; ++j) {
-        const double r_d = row_sum(q_d[j]), r_x = row_sum(q_x[j]);
-        if (lane == 0) {
-            srow[2 * j][row] = r_d;
-            srow[2 * j + 1][row] = r_x;
-        }
+        stats_row_put(srow[2 * j], row, lane, q_d[j]);
+        stats_row_put(srow[2 * j + 1], row, lane, q_x[j]);
     }
-    if (PUSH) {
-        const double r_D = row_sum(q_D);
-        if (lane == 0) srow[2 * NB][row] = r_D;
-    }
+    if (PUSH) stats_row_put(srow[2 * NB], row, lane, q_D);
 }
 template <int NB, bool PUSH>
 __device__ __forceinline__ void multi_stats_finish(double (*srow)[kStatRows + 1], uint32_t nrows, double* partial_delta,
@@ -437,7 +465,7 @@ __device__ __forceinline__ void multi_stats_finish(double (*srow)[kStatRows + 1]
 }
 
 template <class W, int NB, bool PUSH, bool STATS, bool STREAM, int VE, int TPB>
-__global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
+__global__ void __launch_bounds__(TPB, (multi_min_blocks<W, NB, TPB, STATS>()))
 arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
     using T = WTraits<W>;
     const Chunk c = chunks[blockIdx.x];
@@ -464,9 +492,11 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
         nrv = (nvec + 31u) >> 5;
         for (uint32_t vb = warp32; vb < nvec; vb += TPB) {   // a warp walks its rows of 32 vectors together
             const uint32_t v = vb + lane;
-            float q_d[NB], q_x[NB], q_D = 0.f;
+            float q_d[STATS ? NB : 1], q_x[STATS ? NB : 1], q_D = 0.f;   // this thread's items of the row (0 past the end)
+            if (STATS) {
 #pragma unroll
-            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+                for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            }
             if (v < nvec) {
                 const size_t o = (size_t)VE * v;
                 FVec<VE> vh[NB], vs[NB], vx, vm, va;
@@ -502,15 +532,17 @@ arrive_multi_kernel(const Chunk* __restrict__ chunks, ArriveMultiArgs<W> a) {
                     if (STATS) q_D = sumsq<VE>(D);
                 }
             }
-            if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, vb >> 5, lane, q_d, q_x, q_D);
+            if constexpr (STATS) multi_stats_rows<NB, PUSH>(srow, vb >> 5, lane, q_d, q_x, q_D);   // after the stores are out
         }
         done = nvec * VE;
     }
     for (uint32_t ib = done + warp32; ib < c.count; ib += TPB) {
         const uint32_t i = ib + lane;
-        float q_d[NB], q_x[NB], q_D = 0.f;
+        float q_d[STATS ? NB : 1], q_x[STATS ? NB : 1], q_D = 0.f;
+        if (STATS) {
 #pragma unroll
-        for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+        }
         if (i < c.count) {
             float x = th[i], m = ml[i];
 #pragma unroll
@@ -742,7 +774,7 @@ struct ArriveMultiDnArgs {
 };
 
 template <class W, int NB, bool ANYREF, bool PUSH, bool STATS, bool STREAM, int VE, int TPB>
-__global__ void __launch_bounds__(TPB, (NB <= 2 ? 1024 / TPB : (NB <= 4 ? 512 / TPB : 1)))
+__global__ void __launch_bounds__(TPB, (multi_dn_min_blocks<W, NB, TPB, STATS>()))
 arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a) {
     using T = WTraits<W>;
     const Chunk c = chunks[blockIdx.x];
@@ -771,9 +803,11 @@ arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a)
         nrv = (nvec + 31u) >> 5;
         for (uint32_t vb = warp32; vb < nvec; vb += TPB) {
             const uint32_t v = vb + lane;
-            float q_d[NB], q_x[NB], q_D = 0.f;
+            float q_d[STATS ? NB : 1], q_x[STATS ? NB : 1], q_D = 0.f;
+            if (STATS) {
 #pragma unroll
-            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+                for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            }
             if (v < nvec) {
                 const size_t o = (size_t)VE * v;
                 FVec<VE> vh[NB], vs[NB], vx, vc, vm, va;
@@ -825,9 +859,11 @@ arrive_multi_dn_kernel(const Chunk* __restrict__ chunks, ArriveMultiDnArgs<W> a)
     }
     for (uint32_t ib = done + warp32; ib < c.count; ib += TPB) {
         const uint32_t i = ib + lane;
-        float q_d[NB], q_x[NB], q_D = 0.f;
+        float q_d[STATS ? NB : 1], q_x[STATS ? NB : 1], q_D = 0.f;
+        if (STATS) {
 #pragma unroll
-        for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+            for (int j = 0; j < NB; ++j) q_d[j] = q_x[j] = 0.f;
+        }
         if (i < c.count) {
             float x = th[i], acc = ac[i], m = ANYREF ? ml[i] : 0.f;
 #pragma unroll

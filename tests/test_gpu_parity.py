@@ -812,8 +812,12 @@ def test_streaming_replay_keeps_batches_across_calls():
     prod_cut = make(cut)
     for a in range(0, len(events), 5):
         cut.replay(events[a:a + 5], prod_cut, max_batch=8)   # same calls, but every call flushes
-    # streaming fuses as well as one big call and much better than calls that flush
-    assert st.info()["launches"] <= one.info()["launches"] + 1
+    # streaming fuses as well as one big call (except where a call boundary separates a GPS_RECV from the PULL
+    # that directly follows it: those run as two launches instead of one) and much better than calls that flush
+    kinds, lpss = events["kind"], events["lps"]
+    split_pairs = sum(1 for k in range(4, len(events) - 1, 5)
+                      if kinds[k] == tr.GPS_RECV and kinds[k + 1] == tr.PULL and lpss[k] == lpss[k + 1])
+    assert st.info()["launches"] <= one.info()["launches"] + 1 + split_pairs
     assert st.info()["launches"] < 0.9 * cut.info()["launches"]
     log_st = np.concatenate(logs)
     for f in ("kind", "lps", "worker", "t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
