@@ -268,7 +268,8 @@ def run_cpu_table(args):
 # ------------------------------------------------------------------------------------ bandwidth sweep
 def run_sweep(args):
     """Configuration 5: flat fp32 buffers from 2^20 to 2^30 parameters plus the 1.4B-class decoder layout;
-    per size one context with 1 LPS / 1 worker, cycles of {arrive, arrive+due, push, gps, pull}, each kernel
+    per size one context with 1 LPS / 1 worker, cycles of {arrive, arrive+due, push, gps, pull, arrive, arrive+due, push,
+    gps+pull}, each kernel
     timed by the library's CUDA events.  Sizes whose working set is below 512 MB rotate over several
     contexts so that consecutive launches do not find their data in L2."""
     import torch
@@ -303,7 +304,8 @@ def run_sweep(args):
                 h.worker_delta(0, th)
                 assert h.lps_apply(0, 0)
 
-            phases = (a1, a2, lambda h, th: h.lps_push(0), lambda h, th: h.gps_merge(0), lambda h, th: h.lps_pull(0))
+            phases = (a1, a2, lambda h, th: h.lps_push(0), lambda h, th: h.gps_merge(0), lambda h, th: h.lps_pull(0),
+                      a1, a2, lambda h, th: h.lps_push(0), lambda h, th: h.gps_merge_pull(0))
 
             def cycle():
                 # kind-major order: between two launches on the same context all other contexts run,
@@ -324,10 +326,10 @@ def run_sweep(args):
                 for k, (n, ms) in h.timing_read().items():
                     a = agg.setdefault(k, [0, 0.0]); a[0] += n; a[1] += ms
                 h.close()
-            B = {"arrive": 16 + 3 * wb, "push": 12, "gps": 24, "pull": 16}
+            B = {"arrive": 16 + 3 * wb, "push": 12, "gps": 24, "pull": 16, "gps_pull": 36}
             row = {"case": name, "P": P, "tensors": lay.n_tensors, "worker_dtype": wname, "buffer_MB": P * 4 / 1e6,
                    "contexts_rotated": n_sets}
-            for k in ("arrive", "push", "gps", "pull"):
+            for k in ("arrive", "push", "gps", "pull", "gps_pull"):
                 n, ms = agg[k]
                 t = ms / n * 1e-3
                 row[k] = {"us": t * 1e6, "GBps": B[k] * P / 1e9 / t, "frac_of_measured": B[k] * P / 1e9 / t / peak,

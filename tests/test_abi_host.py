@@ -49,6 +49,9 @@ def test_struct_layout_matches_c(tmp_path, lib):
     lines += [f'printf("%zu\\n", offsetof(halos_config, {f}));' for f in fields]
     lines += ['printf("%zu %zu\\n", sizeof(halos_event), sizeof(halos_event_log));',
               'printf("%zu %zu %zu\\n", offsetof(halos_event_log, t), offsetof(halos_event_log, gps_lag), offsetof(halos_event_log, pushed));',
+              'printf("%zu %zu %zu %zu %zu\\n", sizeof(halos_launch_record), offsetof(halos_launch_record, kind), '
+              'offsetof(halos_launch_record, events), offsetof(halos_launch_record, bytes_per_param), offsetof(halos_launch_record, ms));',
+              'printf("%d %d\\n", (int)HALOS_K_COUNT, (int)HALOS_K_GPS_PULL);',
               "return 0;}"]
     src.write_text("\n".join(lines))
     exe = tmp_path / "layout"
@@ -63,6 +66,9 @@ def test_struct_layout_matches_c(tmp_path, lib):
     assert rest[2] == binding.EVENT_LOG_DTYPE.fields["t"][1]
     assert rest[3] == binding.EVENT_LOG_DTYPE.fields["gps_lag"][1]
     assert rest[4] == binding.EVENT_LOG_DTYPE.fields["pushed"][1]
+    lr = binding.LAUNCH_RECORD_DTYPE
+    assert rest[5:10] == [lr.itemsize] + [lr.fields[f][1] for f in ("kind", "events", "bytes_per_param", "ms")]
+    assert rest[10] == len(binding.KERNEL_NAMES) and rest[11] == binding.K_GPS_PULL
     from paper_2506_04531_b200.inputs import trace as tr
     assert tr.EVENT_DTYPE.itemsize == 16 and tr.EVENT_DTYPE.fields["time_ns"][1] == 8
 

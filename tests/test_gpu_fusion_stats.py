@@ -331,3 +331,50 @@ def test_worker_fetch_host_returns_the_scheduled_model(wdt):
         assert np.array_equal(dst.numpy().view(np_dt), want.view(np_dt))
     h.close()
     o.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# per-launch records: kind, events and the algorithmic bytes the library accounts (bench.py's GB/s rest on them)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wdt,wb", [(gen.F32, 4), (gen.BF16, 2)])
+def test_launch_records_account_algorithmic_bytes(wdt, wb):
+    P = 1 << 16
+    init = torch.linspace(-1, 1, P, device="cuda")
+    tdt = torch.float32 if wdt == gen.F32 else torch.int16
+    res = [torch.zeros(P, dtype=tdt, device="cuda") for _ in range(4)]
+    ev = np.zeros(3, dtype=tr.EVENT_DTYPE)
+    ev["worker"] = [0, 1, 2]
+
+    def run(h, fused_window):
+        h.timing_enable(True)
+        h.worker_delta(3, res[3]); h.lps_apply(0, 3)                      # arrive alone
+        h.lps_push(0); h.gps_merge(0); h.lps_pull(0)                        # push, GPS, merge
+        h.replay(ev, lambda i, w, r: res[w], max_batch=8)                   # three arrivals in one launch
+        if fused_window:
+            h.gps_merge_pull(0)                                            # (the batch closed the window)
+        rec = h.timing_launches()
+        return [(hb.KERNEL_NAMES[int(r["kind"])], int(r["events"]), int(r["bytes_per_param"])) for r in rec], rec
+
+    h = hb.Halos(init, [0, 0, 0, 0], worker_dtype=wdt, K=3, **PAPER_HP)     # the merge sets t_last = 1: t = 4 closes the window
+    got, rec = run(h, True)
+    assert got == [("arrive", 1, 16 + 3 * wb), ("push", 0, 12), ("gps", 1, 24), ("pull", 1, 16),
+                   ("arrive_multi", 3, 16 + 9 * wb + 8), ("gps_pull", 2, 36)]
+    assert (rec["ms"] > 0).all() and h.timing_read()["arrive_multi"][0] == 1
+    h.close()
+    # delayed Nesterov, refresh every 2nd LPS update and every 2nd GPS update: +8 bytes where the momentum moves
+    h = hb.Halos(init, [0, 0, 0, 0], worker_dtype=wdt, K=3, **dict(DN_HP, delay_l=2, delay_g=2))
+    got, _ = run(h, True)
+    assert got == [("arrive", 1, 16 + 3 * wb), ("push", 0, 12), ("gps", 1, 24), ("pull", 1, 16),
+                   ("arrive_multi", 3, 16 + 9 * wb + 8 + 8), ("gps_pull", 2, 36 + 8)]
+    h.close()
+    # materialised delta: the arrive reads delta (4 B) instead of theta_H and theta_0
+    h = hb.Halos(init, [0, 0, 0, 0], worker_dtype=wdt, K=100, flags=hb.FLAG_MATERIALISE_DELTA, **PAPER_HP)
+    got, _ = run(h, False)
+    assert got[0] == ("arrive", 1, 20 + wb) and [g[0] for g in got[4:]] == ["arrive"] * 3
+    # new entry points refuse bad arguments without touching the state
+    for call, status in ((lambda: h.gps_merge_pull(7), hb.ERR_INVALID_ARG), (lambda: h.gps_merge_pull(0), hb.ERR_BAD_STATE),
+                         (lambda: h.worker_fetch_host(9, torch.empty(P, dtype=tdt).pin_memory()), hb.ERR_INVALID_ARG)):
+        with pytest.raises(hb.HalosError) as e:
+            call()
+        assert e.value.status == status
+    h.close()
