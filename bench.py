@@ -574,15 +574,17 @@ def run_kernel_table(args):
 
 
 # ------------------------------------------------------------------------------------ shared by both arms
-RESIDENT_BUDGET_BYTES = 137 << 30     # worker results of the timed steps kept in HBM (a B200 has 180 GB; the state needs <= 25 GB)
+DEVICE_BUDGET_BYTES = 160 << 30     # of a B200's 180 GB: the context's state plus the resident worker results of the timed steps
 
 
 def events_per_step(wl, steps: int, asked: int) -> int:
-    """Step length: 128 events unless asked otherwise, cut down so that the results of all timed steps fit the
-    resident budget (~96% of the events are arrivals).  A function of the arguments only, so that both arms
-    of the benchmark replay the same windows."""
+    """Step length: 128 events unless asked otherwise, cut down so that the state and the results of all timed
+    steps fit the device budget (~96% of the events are arrivals).  A function of the arguments only, so that
+    both arms of the benchmark replay the same windows."""
     wbytes = 4 if wl.worker_dtype == 0 else 2
-    fit = RESIDENT_BUDGET_BYTES // (wbytes * wl.layout.P)
+    P = wl.layout.P
+    state = (2 + 5 * wl.n_lps + (1 + wl.n_lps if wl.optimizer else 0)) * 4 * P + wl.n_workers * wbytes * P
+    fit = max(1, (DEVICE_BUDGET_BYTES - state) // (wbytes * P))
     eps = asked if asked > 0 else 128
     return int(max(1, min(eps, (fit * 100 // 96) // max(1, steps))))
 

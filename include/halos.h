@@ -47,7 +47,8 @@ enum {
     HALOS_ERR_BAD_STATE = 2,   /* call order violates Algorithm 1 (e.g. pull before the GPS answered) */
     HALOS_ERR_OOM = 3,
     HALOS_ERR_CUDA = 4,
-    HALOS_ERR_UNSUPPORTED = 5
+    HALOS_ERR_UNSUPPORTED = 5,
+    HALOS_ERR_TIMEOUT = 6      /* reserved for calls that wait on a device-side flag; no call of this build does */
 };
 
 enum { HALOS_F32 = 0, HALOS_BF16 = 1 };
@@ -69,10 +70,10 @@ enum {
     HALOS_FLAG_STATS = 1u,         /* keep per-tensor squared norms of delta, theta_t (arrive) and Delta (push); formed in
                                       registers by the update kernels, in every mode (fused launches, both optimizers,
                                       materialised deltas); needs chunk_elems <= 8192 */
-    HALOS_FLAG_GUARD = 2u,         /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
-    HALOS_FLAG_MATERIALISE_DELTA = 4u  /* halos_worker_delta forms delta (fp32) into a context buffer at once, so the
+    HALOS_FLAG_MATERIALISE_DELTA = 2u, /* halos_worker_delta forms delta (fp32) into a context buffer at once, so the
                                           borrow of theta_H ends when that call has been enqueued; costs one 4P
                                           buffer per worker and 4 + 2 w_b extra bytes of traffic per parameter */
+    HALOS_FLAG_GUARD = 4u          /* surround every state buffer with 256-byte canary zones (halos_check_guards) */
 };
 
 /* LPS phase of the push / merge round trip */

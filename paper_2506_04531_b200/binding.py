@@ -15,11 +15,11 @@ import numpy as np
 _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libhalos_b200.so"
 
-OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED = range(6)
+OK, ERR_INVALID_ARG, ERR_BAD_STATE, ERR_OOM, ERR_CUDA, ERR_UNSUPPORTED, ERR_TIMEOUT = range(7)
 F32, BF16 = 0, 1
 FLAG_STATS = 1
-FLAG_GUARD = 2
-FLAG_MATERIALISE_DELTA = 4
+FLAG_MATERIALISE_DELTA = 2
+FLAG_GUARD = 4
 IDLE, PUSHED, ANSWERED = 0, 1, 2
 BUF_THETA_G, BUF_M_G, BUF_THETA_L, BUF_M_L, BUF_ANCHOR, BUF_OUTBOX, BUF_INBOX, BUF_THETA0, BUF_ACC_L, BUF_ACC_G = range(10)
 OPT_PAPER, OPT_DELAYED_NESTEROV = 0, 1

@@ -1560,6 +1560,7 @@ const char* halos_strerror(int status) {
         case HALOS_ERR_OOM: return "out of memory";
         case HALOS_ERR_CUDA: return "CUDA error";
         case HALOS_ERR_UNSUPPORTED: return "unsupported";
+        case HALOS_ERR_TIMEOUT: return "timed out";
     }
     return "unknown status";
 }

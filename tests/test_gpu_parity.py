@@ -876,9 +876,11 @@ def test_replay_stops_at_the_first_bad_event_and_keeps_what_came_before():
     assert e.value.status == hb.ERR_INVALID_ARG and not asked
     assert not bad.worker_info(0)["pending"]
     # the same for an arrival that would close a window while the previous round trip is still in flight
-    late = hb.Halos(init, [0, 0, 1], K=1, **PAPER_HP)
-    late.replay(ev[:1], lambda i, w, r: res[w])              # K = 1: this arrival pushes
-    with pytest.raises(hb.HalosError) as e:
+    # (the equality test of Alg. 1 line 13 never lets that happen by itself: it takes a push made by hand)
+    late = hb.Halos(init, [0, 0, 1], K=2, **PAPER_HP)
+    late.replay(ev[:1], lambda i, w, r: res[w])              # t = 1
+    late.lps_push(0)                                         # round trip in flight, t_last still 0
+    with pytest.raises(hb.HalosError) as e:                  # t = 2 would close the window of K = 2
         late.replay(ev[2:3], lambda i, w, r: asked.append(w) or res[w])
     assert e.value.status == hb.ERR_BAD_STATE and not asked and not late.worker_info(1)["pending"]
     late.close()
