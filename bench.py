@@ -345,8 +345,8 @@ def run_sweep(args):
 def pcie_ceiling(torch, dev, nbytes: int, reps: int = 6):
     """Pinned host<->device copies of one result's size, both directions at once on two streams (the shape of the
     end-to-end leg): GB/s per direction.  Plain cudaMemcpyAsync through torch, no library code."""
-    hin = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
-    hout = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    hin = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    hout = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
     din = torch.empty(nbytes, dtype=torch.uint8, device=dev)
     dout = torch.empty(nbytes, dtype=torch.uint8, device=dev)
     s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
@@ -384,9 +384,9 @@ def run_e2e(args, wl, hb, tr, torch, dist, dev, fresh_context, timed_events, arr
     per_step = max(1, sum(1 for i in arrive_slots if i < eps))
     steps = int(max(1, min(K, budget // (wbytes * P) // per_step)))
     n_arr = sum(1 for i in arrive_slots if i < steps * eps)
-    host_results = torch.empty((n_arr, P), dtype=wdt).pin_memory()
+    host_results = torch.empty((n_arr, P), dtype=wdt, pin_memory=True)   # allocated pinned: no pageable twin
     host_results.copy_(resident[:n_arr])
-    ring = [torch.empty(P, dtype=wdt).pin_memory() for _ in range(4)]   # answers: a worker consumes its own at once
+    ring = [torch.empty(P, dtype=wdt, pin_memory=True) for _ in range(4)]   # answers: a worker consumes its own at once
     ceiling = pcie_ceiling(torch, dev, wbytes * P)
     h = fresh_context()
     torch.cuda.synchronize(dev)
