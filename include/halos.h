@@ -226,7 +226,9 @@ typedef int (*halos_producer_fn)(void* user, uint32_t event_index, uint32_t work
  * K closes, fused into the same launch), GPS_RECV = gps_merge, PULL = lps_pull (with max_batch > 1, a
  * GPS_RECV directly followed by the PULL of the same LPS runs as halos_gps_merge_pull).  log_host (may be
  * NULL) receives one record per event.  Stops at the first failing event: returns its status and
- * writes its index to *failed_at (may be NULL); events before it stay applied. */
+ * writes its index to *failed_at (may be NULL); events before it stay applied.  An ARRIVE that cannot be
+ * applied (worker of another LPS; window due while a round trip is in flight) is refused BEFORE the
+ * producer is asked, so a failed replay never leaves a borrowed result registered. */
 int halos_replay(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                  void* user, halos_event_log* log_host, uint32_t* failed_at);
 
