@@ -378,3 +378,47 @@ def test_launch_records_account_algorithmic_bytes(wdt, wb):
             call()
         assert e.value.status == status
     h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# randomised equivalence: any split into streaming calls, any batch limit, both optimizers and
+# worker dtypes -- the fused driver leaves the state and the log of the per-event replay
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(8))
+def test_fused_driver_equals_per_event_replay_on_random_traces(seed):
+    rng = np.random.default_rng(900 + seed)
+    n_lps = int(rng.integers(1, 4))
+    n_workers = int(rng.integers(n_lps, 11))
+    worker_lps = [int(x) for x in np.concatenate([np.arange(n_lps), rng.integers(0, n_lps, n_workers - n_lps)])]
+    K = int(rng.integers(1, 7))
+    wdt = gen.BF16 if seed % 2 else gen.F32
+    dn = seed % 4 >= 2
+    hp = dict(DN_HP, K=K, delay_l=int(rng.integers(1, 5)), delay_g=int(rng.integers(1, 4))) if dn else dict(PAPER_HP, K=K)
+    sizes = [int(x) for x in rng.integers(1, 9000, size=int(rng.integers(1, 7)))]
+    lay = layouts.ragged_layout("r", sizes)
+    events = tr.random_trace(worker_lps, 220, K, seed=seed)
+    dg = DeviceGenerator(lay, 300 + seed)
+    mk = lambda: hb.Halos(dg.theta_init(), worker_lps, lay.numel, worker_dtype=wdt, chunk_elems=int(rng.choice([256, 1024, 4096])),
+                          flags=hb.FLAG_GUARD, **hp)
+    ref = mk()
+    log_ref = ref.replay(events, _producer(ref, dg, lay, worker_lps, wdt))
+    fus = mk()
+    prod = _producer(fus, dg, lay, worker_lps, wdt)
+    logs, pos = [], 0
+    while pos < len(events):                     # random call lengths, random batch limits, streaming or flushing calls
+        n = int(rng.integers(1, 40))
+        logs.append(fus.replay(events[pos:pos + n], prod, max_batch=int(rng.integers(2, 9)), keep_queued=bool(rng.integers(0, 2))))
+        pos += n
+    fus.flush()
+    log_fus = np.concatenate(logs)
+    extra = [hb.BUF_ACC_L, hb.BUF_ACC_G] if dn else []
+    _same_state(ref, fus, n_workers, n_lps, ALL_BUFS + extra)
+    for f in ("kind", "lps", "worker", "t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+        assert np.array_equal(log_ref[f], log_fus[f]), f
+    for l in range(n_lps):
+        assert ref.counters(l) == fus.counters(l)
+    assert fus.check_guards() == -1 and ref.check_guards() == -1
+    assert fus.info()["launches"] <= ref.info()["launches"]
+    assert int(log_fus["fused"].sum()) > 0
+    ref.close()
+    fus.close()
