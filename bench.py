@@ -775,11 +775,17 @@ def main():
 
     peak, peak_kind = measured_peak_gbs()
 
-    def timed_region(max_batch):
-        """K timed steps from the state after the warm-up, reading the resident results."""
+    # per step: the table of result pointers of its events (the resident results), built once outside the timed regions
+    step_tables = [hb.result_table(timed_events[s * eps:(s + 1) * eps],
+                                   [resident[arrive_slots[s * eps + k]] if (s * eps + k) in arrive_slots else None for k in range(eps)])
+                   for s in range(K)]
+
+    def timed_region(max_batch, instrumented=True):
+        """K timed steps from the state after the warm-up, reading the resident results.  instrumented: the library
+        brackets every launch with CUDA events (per-kernel durations; costs ~4 us per launch)."""
         h = fresh_context()
         torch.cuda.synchronize(dev)
-        h.timing_enable(True)
+        h.timing_enable(instrumented)
         launches0 = h.info()["launches"]
         if world > 1:
             dist.barrier()
@@ -789,10 +795,10 @@ def main():
             e0.record()
             for s in range(K):
                 base = s * eps
-                # streaming form: arrivals still waiting for companions at the end of a step may be fused
-                # with arrivals of the next step; everything is launched before the region ends
-                h.replay(timed_events[base:base + eps], lambda index, worker, rnd, base=base: resident[arrive_slots[base + index]],
-                         want_log=False, max_batch=max_batch, keep_queued=True)
+                # the results exist already: table-driven replay (no Python per event).  Streaming form: arrivals still
+                # waiting for companions at the end of a step may be fused with arrivals of the next step; everything
+                # is launched before the region ends
+                h.replay_results(timed_events[base:base + eps], step_tables[s], want_log=False, max_batch=max_batch, keep_queued=True)
             h.flush()
             e1.record()
             torch.cuda.synchronize(dev)
@@ -807,6 +813,8 @@ def main():
         h.close()
         units = float(K * eps) * P
         t_ms, units_all = reduce_over_ranks(dist if world > 1 else None, elapsed_ms, units, dev)
+        if not instrumented:
+            return {"value": units_all / (t_ms * 1e-3), "ms_per_step": t_ms / K, "launches": int(launches)}
         per_kernel = kernel_table(records, P, elapsed_ms)
         dominant = max(per_kernel, key=lambda k: (per_kernel[k]["share_of_step"] or 0))
         d = per_kernel[dominant]
@@ -829,6 +837,10 @@ def main():
                          "dominant_kernel_GBps": spread([r["roofline"]["achieved"] for r in runs])}
         reasons = sorted({x for r in runs for x in r["clocks"]["reasons"]})
         med["clocks"] = dict(med["clocks"], reasons=reasons)
+        # the same region without the per-launch events: what the instrumentation costs
+        plain = sorted((timed_region(max_batch, instrumented=False) for _ in range(3)), key=lambda r: r["value"])[1]
+        med["uninstrumented"] = {"value": plain["value"], "unit": UNIT, "ms_per_step": plain["ms_per_step"],
+                                 "note": "same region, per-launch CUDA events off (median of 3)"}
         return med
 
     per_event = repeated(1)                               # one kernel per event: the per-event figure of the metric
@@ -881,13 +893,14 @@ def main():
                 "warmup": args.warmup, "ms_per_step": per_event["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
                 "clocks": per_event["clocks"], "e2e": e2e, "gpu_launches": per_event["launches"],
-                "roofline": per_event["roofline"], "spread": per_event["spread"], "cpu_baseline": cpu,
+                "roofline": per_event["roofline"], "spread": per_event["spread"], "uninstrumented": per_event["uninstrumented"],
+                "cpu_baseline": cpu,
                 "note": "value = one kernel launch per event (the per-event figure of the metric); fused_replay = the same "
                         "events through the driver's multi-event fusion (bit-identical state, fewer bytes per event)"}
         if fused is not None:
             line["fused_replay"] = {"value": fused["value"], "unit": UNIT, "ms_per_step": fused["ms_per_step"],
                                     "gpu_launches": fused["launches"], "roofline": fused["roofline"], "spread": fused["spread"],
-                                    "clocks": fused["clocks"]}
+                                    "uninstrumented": fused["uninstrumented"], "clocks": fused["clocks"]}
         if configs is not None:
             line["configs"] = configs
         print(json.dumps(line))

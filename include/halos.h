@@ -256,6 +256,17 @@ int halos_replay_batched(halos_ctx* ctx, const halos_event* events_host, uint32_
 int halos_replay_stream(halos_ctx* ctx, const halos_event* events_host, uint32_t n, halos_producer_fn producer,
                         void* user, halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch);
 
+/* The same drivers for results that already exist (a stored trace replayed with its stored results, or a
+ * backlog of results that arrived while the server was busy): results_host[k] is the flat device pointer
+ * (P elements of worker_dtype) of event k if it is an ARRIVE and ignored otherwise; no callback is made.
+ * keep_queued = 0 behaves like halos_replay_batched, nonzero like halos_replay_stream; the borrow rules are
+ * those of the respective call (a result must stay valid until the same worker's next arrival has been
+ * launched, the replay has returned, or -- streaming -- halos_flush).  A NULL entry for an ARRIVE fails
+ * that event with INVALID_ARG.  The host cost per event is one kernel launch at most, which matters for
+ * models small enough to be launch-bound. */
+int halos_replay_results(halos_ctx* ctx, const halos_event* events_host, uint32_t n, const void* const* results_host,
+                         halos_event_log* log_host, uint32_t* failed_at, uint32_t max_batch, int keep_queued);
+
 /* Launches every arrival that halos_replay_stream left queued. */
 int halos_flush(halos_ctx* ctx);
 

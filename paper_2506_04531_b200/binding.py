@@ -34,7 +34,7 @@ EXPORTED = (
     "halos_timing_read", "halos_strerror", "halos_last_error", "halos_push_noalloc", "halos_export_file",
     "halos_import_file", "halos_replay_batched", "halos_batch_info", "halos_check_guards", "halos_replay_stream",
     "halos_flush", "halos_gps_merge_pull", "halos_stats_log", "halos_worker_fetch_host", "halos_fetch_sync",
-    "halos_timing_launches",
+    "halos_timing_launches", "halos_replay_results",
 )
 NOALLOC_MAX_ELEMS = 1 << 29
 
@@ -110,6 +110,7 @@ def load_library():
     lib.halos_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.halos_replay_stream.argtypes = [vp, vp, u32, PRODUCER_FN, vp, vp, C.POINTER(u32), u32]
     lib.halos_flush.argtypes = [vp]
+    lib.halos_replay_results.argtypes = [vp, vp, u32, vp, vp, C.POINTER(u32), u32, i32]
     lib.halos_batch_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
     lib.halos_peek.argtypes = [vp, u32, u32, C.POINTER(vp), C.POINTER(u64)]
     lib.halos_read.argtypes = [vp, u32, u32, u64, u64, vp]
@@ -160,6 +161,12 @@ def push_noalloc(theta, anchor, Delta_out, sqnorm_out, n=None, stream=None) -> i
     dev = theta.device.index if hasattr(theta, "device") and theta.device.index is not None else torch.cuda.current_device()
     st = (stream if stream is not None else torch.cuda.current_stream(dev)).cuda_stream
     return int(lib.halos_push_noalloc(dev, st, _ptr(theta), _ptr(anchor), _ptr(Delta_out), n, _ptr(sqnorm_out)))
+
+
+def result_table(events: np.ndarray, results):
+    """The pointer table halos_replay_results takes: entry k = address of results[k] for ARRIVE events, NULL otherwise.
+    Build it once for a window that is replayed through ``Halos.replay_results`` (keep the tensors alive yourself)."""
+    return (C.c_void_p * len(events))(*[(_ptr(r) if int(k) == EV_ARRIVE else None) for r, k in zip(results, events["kind"])])
 
 
 class Halos:
@@ -352,6 +359,23 @@ class Halos:
                 log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch))
         if err:
             raise err[0]
+        if rc != OK:
+            raise HalosError(rc, f"event {failed.value}: " + self._lib.halos_last_error(self._h).decode())
+        return log
+
+    def replay_results(self, events: np.ndarray, results, want_log: bool = True, max_batch: int = 1,
+                       keep_queued: bool = False):
+        """replay() for results that already exist: ``results[k]`` is the flat CUDA tensor (or address) of event k if
+        it is an ARRIVE (anything else is ignored there).  No Python code runs per event.  The tensors must stay
+        alive and unchanged until their kernels have run (with keep_queued: until flush())."""
+        ev = np.ascontiguousarray(events)
+        assert ev.dtype.itemsize == C.sizeof(Event) and len(results) == len(ev)
+        table = results if isinstance(results, C.Array) else result_table(ev, results)
+        log = np.zeros(len(ev), dtype=EVENT_LOG_DTYPE) if want_log else None
+        failed = C.c_uint32(0)
+        rc = self._lib.halos_replay_results(self._h, ev.ctypes.data, len(ev), table,
+                                            log.ctypes.data if log is not None else None, C.byref(failed), int(max_batch),
+                                            int(bool(keep_queued)))
         if rc != OK:
             raise HalosError(rc, f"event {failed.value}: " + self._lib.halos_last_error(self._h).decode())
         return log

@@ -1221,6 +1221,21 @@ int halos_replay_batched(halos_ctx* c, const halos_event* ev, uint32_t n, halos_
     return rc != HALOS_OK ? rc : rf;
 }
 
+// Producer over a table of results: entry k is the flat result of event k (ARRIVE events only).
+static int table_producer(void* user, uint32_t event_index, uint32_t, uint64_t, const void** flat_dev, const void* const**) {
+    *flat_dev = static_cast<const void* const*>(user)[event_index];
+    return *flat_dev ? 0 : 1;
+}
+
+int halos_replay_results(halos_ctx* c, const halos_event* ev, uint32_t n, const void* const* results_host, halos_event_log* log,
+                         uint32_t* failed_at, uint32_t max_batch, int keep_queued) {
+    if (!c) return HALOS_ERR_INVALID_ARG;
+    if (n && !results_host) return fail(c, HALOS_ERR_INVALID_ARG, "null result table");
+    void* user = const_cast<void*>(static_cast<const void*>(results_host));
+    return keep_queued ? halos_replay_stream(c, ev, n, table_producer, user, log, failed_at, max_batch)
+                       : halos_replay_batched(c, ev, n, table_producer, user, log, failed_at, max_batch);
+}
+
 int halos_replay(halos_ctx* c, const halos_event* ev, uint32_t n, halos_producer_fn producer, void* user,
                  halos_event_log* log, uint32_t* failed_at) {
     return halos_replay_batched(c, ev, n, producer, user, log, failed_at, 1);

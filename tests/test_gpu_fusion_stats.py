@@ -422,3 +422,48 @@ def test_fused_driver_equals_per_event_replay_on_random_traces(seed):
     assert int(log_fus["fused"].sum()) > 0
     ref.close()
     fus.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# table-driven replay (results that already exist, no callback) = replay with a producer
+# ---------------------------------------------------------------------------------------------
+def test_replay_results_equals_replay_with_a_producer():
+    lay = layouts.ragged_layout("r", [4099, 33, 20001, 5, 8192])
+    worker_lps = [0, 0, 0, 1, 1]
+    hp = dict(PAPER_HP, K=4)
+    events = tr.random_trace(worker_lps, 120, 4, seed=21)
+    dg = DeviceGenerator(lay, 61)
+    ref = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+    kept = []                                                # every result of the reference run, in event order
+
+    def producer(index, worker, rnd):
+        r = dg.worker_result(ref.peek(hb.BUF_THETA0, worker), worker, rnd)
+        kept.append((index, r))
+        return r
+    log_ref = ref.replay(events, producer)
+    results = [None] * len(events)
+    for index, r in kept:
+        results[index] = r
+    for mb, streaming in ((1, False), (8, False), (8, True)):
+        h = hb.Halos(dg.theta_init(), worker_lps, lay.numel, chunk_elems=1024, **hp)
+        if streaming:
+            logs = [h.replay_results(events[a:a + 7], results[a:a + 7], max_batch=mb, keep_queued=True) for a in range(0, len(events), 7)]
+            h.flush()
+            log = np.concatenate(logs)
+        else:
+            log = h.replay_results(events, hb.result_table(events, results), max_batch=mb)
+        _same_state(ref, h, len(worker_lps), 2)
+        for f in ("kind", "lps", "worker", "t", "t_last", "gps_iter", "worker_staleness", "gps_lag", "pushed"):
+            assert np.array_equal(log_ref[f], log[f]), f
+        h.close()
+    # an ARRIVE without a result fails that event and leaves nothing registered
+    h = hb.Halos(dg.theta_init(), worker_lps, lay.numel, **hp)
+    first = int(np.nonzero(events["kind"] == tr.ARRIVE)[0][1])
+    broken = list(results)
+    broken[first] = None
+    with pytest.raises(hb.HalosError) as e:
+        h.replay_results(events, broken)
+    assert e.value.status == hb.ERR_INVALID_ARG and f"event {first}" in str(e.value)
+    assert not h.worker_info(int(events["worker"][first]))["pending"]
+    h.close()
+    ref.close()
