@@ -385,8 +385,9 @@ arrive_kernel(const Chunk* __restrict__ chunks, ArriveArgs<W> a) {
 // and momentum are read and written once for the whole batch; per element the NB updates are applied
 // in queue order in registers, so the result is bit-identical to NB single launches.  Traffic per
 // batch: 8 + 8 (theta, m read + write) + NB x (2 w_b read + w_b write) instead of NB x (16 + 3 w_b).
-// Only the last arrival of a batch may close a window of K (PUSH).  Batches of up to 4 run with the
-// regular CTA size; 5..8 need ~150 registers per thread and run with 256-thread CTAs.
+// Only the last arrival of a batch may close a window of K (PUSH).  Batches of 2 run with the regular CTA
+// size (512 threads, 2 CTAs per SM); batches of 3..8 with 256-thread CTAs: 2 per SM up to 4 arrivals, and
+// for 5..8 (150-240 registers with fp32 results) one per SM -- two for bf16 results, see multi_min_blocks.
 // =====================================================================================================
 constexpr int kMaxBatch = 8;
 constexpr int kMultiWideThreads = 256;   // CTA size of the multi-arrival kernel for batches of 3..8 (register budget)
