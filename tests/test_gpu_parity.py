@@ -678,9 +678,10 @@ def test_api_fuzz_statuses_and_state(seed):
     pending = {}                                # worker -> result (numpy) registered but not applied
     keep = {}
     phase = [hb.IDLE] * n_lps
+    fetched = []
     n_ok = n_bad = 0
     for step in range(700):
-        op = int(rng.integers(0, 5))
+        op = int(rng.integers(0, 7))
         l, w = int(rng.integers(0, n_lps + 1)), int(rng.integers(0, len(worker_lps) + 1))   # sometimes out of range
         if rng.random() < 0.85:                 # mostly well-formed arguments, so that the state really advances
             l, w = min(l, n_lps - 1), min(w, 4)
@@ -715,12 +716,25 @@ def test_api_fuzz_statuses_and_state(seed):
             if want == hb.OK:
                 o.gps_recv(l)
                 phase[l] = hb.ANSWERED
-        else:
+        elif op == 4:
             call = lambda: h.lps_pull(l)
             want = hb.ERR_INVALID_ARG if l >= n_lps else (hb.ERR_BAD_STATE if phase[l] != hb.ANSWERED else hb.OK)
             if want == hb.OK:
                 o.pull(l)
                 phase[l] = hb.IDLE
+        elif op == 5:                           # GPS update and merge as one launch
+            call = lambda: h.gps_merge_pull(l)
+            want = hb.ERR_INVALID_ARG if l >= n_lps else (hb.ERR_BAD_STATE if phase[l] != hb.PUSHED else hb.OK)
+            if want == hb.OK:
+                o.gps_recv(l)
+                o.pull(l)
+                phase[l] = hb.IDLE
+        else:                                   # the worker's start model copied out while later updates run on
+            dst = torch.empty(lay.P, dtype=torch.float32).pin_memory()
+            call = lambda: h.worker_fetch_host(w, dst)
+            want = hb.ERR_INVALID_ARG if w >= 5 else hb.OK
+            if want == hb.OK:
+                fetched.append((dst, o.buffer("th0", w).copy()))
         if want == hb.OK:
             call()
             n_ok += 1
@@ -730,6 +744,10 @@ def test_api_fuzz_statuses_and_state(seed):
             assert e.value.status == want, (step, op, l, w)
             n_bad += 1
     assert n_ok > 150 and n_bad > 150
+    h.fetch_sync()
+    assert len(fetched) > 20
+    for dst, want_th0 in fetched:
+        assert np.array_equal(dst.numpy().view(np.uint32), want_th0.view(np.uint32))
     for l in range(n_lps):
         assert h.counters(l) == o.counters(l)
         for which, name in ((hb.BUF_THETA_L, "th"), (hb.BUF_M_L, "ml"), (hb.BUF_ANCHOR, "anchor"),
